@@ -1,0 +1,191 @@
+/*
+ * patdnn.h -- C ABI of the pattern-sparse 3x3 convolution library (NVIDIA B200, sm_100a).
+ *
+ * The operation is the inference hot path of PatDNN (Niu et al., ASPLOS 2020): a 3x3, stride-1, pad-1
+ * convolution whose weights satisfy the two constraint sets of Section 4.2 (Eq. 1) --
+ *   kernel pattern pruning : every kept (filter, channel) kernel keeps exactly 4 of its 9 weights, at the
+ *                            positions of one pattern out of a small fixed set;
+ *   connectivity pruning   : whole (filter, channel) kernels are removed.
+ * The host side builds the compressed weight storage of Section 5.3 (FKW: offset, reorder, index, stride and
+ * weight arrays) after the filter-kernel reorder of Section 5.2 (FKR); the device side runs the branch-free,
+ * pattern-specialised, register-reusing loops of Sections 5.2 and 5.4 with a fused bias + ReLU epilogue.
+ *
+ * Conventions used by every call
+ *   - tap t = 3*r + s (r = kernel row, s = kernel column); a pattern is a 9-bit mask, bit t set = tap t kept,
+ *     exactly four bits set; the pattern id of a kernel is the 0-based position of its mask in `pattern_set`.
+ *   - tensors are dense, row-major, NCHW / OIHW; the output has the input's spatial size.
+ *   - out[n,f,y,x] = act(bias[f] + sum_{c,r,s} (weights*mask)[f,c,r,s] * in[n,c,y+r-1,x+s-1]), input = 0 outside
+ *     the image, act = max(0,.) when `relu` is set (cross-correlation, no kernel flip).
+ *   - every function returns a status code (0 = PATDNN_OK); nothing aborts, throws or prints.
+ *   - pointers are marked HOST or DEVICE; the library never frees or keeps a caller pointer after the call
+ *     returns, except where a stack keeps the handles it was built from.
+ *   - there is no CPU fallback: the compute entry points fail with PATDNN_E_CUDA / PATDNN_E_NO_DEVICE when no
+ *     usable device is present.
+ */
+#ifndef PATDNN_H
+#define PATDNN_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define PATDNN_API __attribute__((visibility("default")))
+#else
+#define PATDNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PATDNN_OK = 0,
+    PATDNN_E_NULL = 1,          /* a required pointer is NULL */
+    PATDNN_E_SHAPE = 2,         /* a size is non-positive, too large, or unsupported */
+    PATDNN_E_PATTERN_SET = 3,   /* a pattern does not have exactly 4 of 9 bits, is duplicated, or P is not in 1..32 */
+    PATDNN_E_MASK = 4,          /* a kernel's mask is neither empty nor a pattern of the set (Section 4.2) */
+    PATDNN_E_ORDER = 5,         /* caller-supplied filter order is not a permutation */
+    PATDNN_E_CUDA = 6,          /* a CUDA call failed; patdnn_last_cuda_error() has the text */
+    PATDNN_E_NO_DEVICE = 7,     /* handle was encoded host-only, or no CUDA device is usable */
+    PATDNN_E_DEVICE_TIMEOUT = 8,/* a bounded device-side wait expired */
+    PATDNN_E_DTYPE = 9,         /* unknown dtype / variant value */
+    PATDNN_E_ALLOC = 10,        /* host allocation failed */
+    PATDNN_E_STACK = 11         /* layers of a stack do not chain (shape or dtype mismatch) */
+};
+
+enum { PATDNN_F32 = 0, PATDNN_F16 = 1 };   /* storage type of weights and activations; accumulation is fp32 */
+
+/* Kernel variants.  AUTO picks the tiled kernel planned for the layer's shape; the others exist for the ablation
+ * ladder of Section 6.3 (no optimisation -> +reorder -> +load-redundancy elimination). */
+enum {
+    PATDNN_VARIANT_AUTO = 0,
+    PATDNN_VARIANT_NOOPT = 1,     /* original filter order, per-kernel branch on the pattern, global loads */
+    PATDNN_VARIANT_REORDER = 2,   /* walks the FKW arrays in pattern order (branch-free per run), global loads */
+    PATDNN_VARIANT_TILED = 3      /* shared-memory tile + halo, register patch reuse across taps and filters */
+};
+
+enum { PATDNN_FLAG_HOST_ONLY = 1 };   /* encode on the host only: no device is touched, patdnn_conv is refused */
+
+typedef struct patdnn_layer *patdnn_handle;   /* opaque; owned by the library until patdnn_free */
+typedef struct patdnn_stack_s *patdnn_stack;  /* opaque; owned by the library until patdnn_stack_free */
+
+typedef struct {
+    int32_t F, C;            /* filters (output channels), input channels; kernel 3x3, stride 1, pad 1 */
+    int32_t N, H, W;         /* batch and spatial size the handle is planned for */
+    int32_t dtype;           /* PATDNN_F32 or PATDNN_F16 */
+    int32_t relu;            /* 1 = fuse ReLU after the bias add */
+    int32_t filter_order;    /* 0 = filter reorder of Section 5.2; 1 = caller-supplied order (kernel reorder still applies) */
+    const int32_t *order;    /* HOST [F] permutation (position -> original filter) when filter_order == 1, else NULL */
+    const float *bias;       /* HOST [F] in original filter numbering, or NULL for zeros */
+    int32_t variant;         /* PATDNN_VARIANT_* */
+    int32_t flags;           /* PATDNN_FLAG_* */
+} patdnn_desc;
+
+/*
+ * patdnn_encode -- validate a pruned layer against its pattern set (Section 4.2), run the filter-kernel reorder
+ * (Section 5.2), build the FKW arrays (Section 5.3), derive the private device layout and upload it.
+ *   weights      HOST float  [F][C][3][3]; values where mask == 0 are ignored; a kept weight may be 0.0
+ *   mask         HOST uint8  [F][C][3][3], entries 0 or 1
+ *   pattern_set  HOST uint16 [n_patterns] 9-bit masks, 1 <= n_patterns <= 32
+ *   desc         HOST; copied
+ *   out          receives the handle on success (untouched on failure)
+ * Errors: E_NULL, E_SHAPE, E_PATTERN_SET, E_MASK, E_ORDER, E_DTYPE, E_ALLOC, E_CUDA.
+ * The call is synchronous (it returns after the upload completed) and uses the current CUDA device.
+ */
+PATDNN_API int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pattern_set, int32_t n_patterns,
+                  const patdnn_desc *desc, patdnn_handle *out);
+
+/*
+ * patdnn_conv -- run the layer (Sections 5.2 and 5.4: pattern-ordered branch-free loops with load-redundancy
+ * elimination; bias + ReLU fused) asynchronously on `stream`.
+ *   in   DEVICE [N][C][H][W] of the handle's dtype (float or IEEE half), 16-byte aligned
+ *   out  DEVICE [N][F][H][W] of the same dtype, 16-byte aligned; must not overlap `in`
+ *   stream  a cudaStream_t (NULL = default stream).  No synchronisation happens inside.
+ * Errors: E_NULL, E_NO_DEVICE, E_CUDA (launch failure).
+ */
+PATDNN_API int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream);
+
+/*
+ * patdnn_conv_host -- the same operation with HOST buffers: copies `in` to a handle-owned device buffer, runs the
+ * layer, copies the result back, all on `stream`, and waits for the stream before returning.  Pinned host memory
+ * makes the copies asynchronous with respect to other streams.  The device buffers are allocated on first use and
+ * live until patdnn_free.
+ */
+PATDNN_API int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void *stream);
+
+/* patdnn_free -- release the handle and everything it owns (device and host).  NULL is accepted. */
+PATDNN_API int patdnn_free(patdnn_handle h);
+
+/* Canonical FKW arrays (Section 5.3), HOST memory owned by the handle and valid until patdnn_free.
+ *   offset  [F+1] kernels stored before filter position i; offset[F] = K
+ *   reorder [F]   original output channel of the filter at position i
+ *   index   [K]   input channel of stored kernel k
+ *   stride  [F][P+1] per filter, cumulative kernel counts per pattern (stride[i][0] = 0, stride[i][P] = length)
+ *   weight  [K][4] the kept weights in ascending tap order: float (F32) or IEEE half bit patterns (F16, uint16)
+ * Order inside a filter: ascending pattern id, then ascending input channel.  Filter order: ascending length; inside
+ * one length a greedy chain from the smallest original id to the most similar unplaced filter (ties: smallest id).
+ */
+typedef struct {
+    int32_t F, C, P, K;
+    const int32_t *offset;
+    const int32_t *reorder;
+    const int32_t *index;
+    const int32_t *stride;
+    const void *weight;
+} patdnn_fkw_view;
+
+/* patdnn_export -- fill `v` with pointers to the handle's canonical FKW arrays (no copy). */
+PATDNN_API int patdnn_export(patdnn_handle h, patdnn_fkw_view *v);
+
+/* patdnn_decode -- rebuild dense HOST float [F][C][3][3] weights from the FKW arrays; equals weights*mask bit for
+ * bit for F32 handles and the half-rounded values for F16 handles. */
+PATDNN_API int patdnn_decode(patdnn_handle h, float *dense_out);
+
+/* Planned launch geometry of a handle, for reports and tests. */
+typedef struct {
+    int32_t variant;            /* resolved PATDNN_VARIANT_* */
+    int32_t tile_rows, tile_cols;   /* output pixels per thread (rows x columns) */
+    int32_t filters_per_warp;   /* register-blocked filters sharing one input patch */
+    int32_t warps_per_cta;
+    int32_t channels_per_stage; /* input channels staged per shared-memory buffer */
+    int32_t channel_splits;     /* >1: the channel range is split across a thread-block cluster */
+    int32_t grid_x, grid_y, grid_z;
+    int32_t smem_bytes;
+    int64_t device_bytes;       /* bytes of the private device layout */
+    int64_t entries;            /* kernel entries in the device layout (kept kernels plus padding) */
+} patdnn_plan_info;
+
+PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
+
+/*
+ * A stack chains layers on the device: layer i's output is layer i+1's input, optionally through a 2x2/stride-2
+ * max-pool (the VGG-16 arrangement).  The stack owns two ping-pong activation buffers; the handles stay owned by
+ * the caller and must outlive the stack.
+ *   patdnn_stack_create   handles HOST [n]; pool_after HOST [n] (1 = max-pool after that layer) or NULL
+ *   patdnn_stack_run      in DEVICE [N][C0][H0][W0]; out DEVICE, the last layer's (pooled) output; asynchronous
+ *   patdnn_stack_run_host the same with HOST buffers; copies in, runs, copies out, waits for the stream
+ *   patdnn_stack_out_shape  N, F, H, W of the stack's output
+ * Errors: E_NULL, E_STACK, E_CUDA, E_NO_DEVICE.
+ */
+PATDNN_API int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after, int32_t n, patdnn_stack *out);
+PATDNN_API int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream);
+PATDNN_API int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
+PATDNN_API int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, int32_t *W);
+PATDNN_API int patdnn_stack_free(patdnn_stack s);
+
+/* patdnn_maxpool2x2 -- 2x2 / stride-2 max-pool (floor) on DEVICE NCHW tensors of the given dtype; asynchronous.
+ * Not part of the paper's method; provided so that the VGG-shaped stack runs without any other library. */
+PATDNN_API int patdnn_maxpool2x2(const void *in, void *out, int32_t N, int32_t C, int32_t H, int32_t W, int32_t dtype,
+                      void *stream);
+
+/* Number of this library's kernels launched on the calling thread's behalf since the last reset (for reports). */
+PATDNN_API int64_t patdnn_launch_count(void);
+PATDNN_API void patdnn_reset_launch_count(void);
+
+PATDNN_API const char *patdnn_strerror(int status);
+PATDNN_API const char *patdnn_last_cuda_error(void);   /* text of the last CUDA failure seen by this thread ("" if none) */
+PATDNN_API const char *patdnn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PATDNN_H */

@@ -1,0 +1,401 @@
+// C ABI of the library (declared in include/patdnn.h): handles, uploads, launches.  No torch types anywhere.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/patdnn.h"
+#include "fkw_encoder.hpp"
+#include "kernels.hpp"
+
+using namespace patdnn;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+std::atomic<int64_t> g_launches{0};
+
+int cuda_fail(cudaError_t e, const char *what) {
+    g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    cudaGetLastError();                       // clear the sticky-free error state
+    return PATDNN_E_CUDA;
+}
+#define CU(call)                                             \
+    do {                                                     \
+        cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);  \
+    } while (0)
+
+template <typename T>
+int upload(const std::vector<T> &v, T **dptr, std::vector<void *> &owned) {
+    *dptr = nullptr;
+    const size_t bytes = std::max<size_t>(v.size() * sizeof(T), 16);
+    void *d = nullptr;
+    CU(cudaMalloc(&d, bytes));
+    owned.push_back(d);
+    if (!v.empty()) CU(cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
+    *dptr = static_cast<T *>(d);
+    return PATDNN_OK;
+}
+
+}  // namespace
+
+struct patdnn_layer {
+    patdnn_desc desc{};
+    Fkw fkw;
+    std::vector<float> bias;                 // [F], zeros if the caller gave none
+    int variant = PATDNN_VARIANT_REORDER;    // resolved
+    bool on_device = false;
+    int device = -1;
+    std::vector<void *> owned;               // device allocations
+    // canonical arrays on the device
+    int32_t *d_offset = nullptr, *d_reorder = nullptr, *d_index = nullptr, *d_stride = nullptr;
+    int32_t *d_kernel_pid = nullptr, *d_dense_slot = nullptr;
+    float *d_weight = nullptr, *d_bias = nullptr;
+    uint16_t *d_patterns = nullptr;
+    // tiled kernel
+    TiledPlan plan;
+    uint32_t *d_desc = nullptr;
+    float *d_wts = nullptr;
+    int32_t *d_seg = nullptr, *d_seglen = nullptr;
+    int64_t device_bytes = 0;
+    // staging buffers of patdnn_conv_host
+    void *d_in_stage = nullptr, *d_out_stage = nullptr;
+};
+
+struct patdnn_stack_s {
+    std::vector<patdnn_handle> layers;
+    std::vector<int32_t> pool;
+    void *buf[2] = {nullptr, nullptr};
+    void *d_in = nullptr, *d_out = nullptr;   // staging buffers of patdnn_stack_run_host
+    size_t buf_bytes = 0, in_bytes = 0, out_bytes = 0;
+    int32_t oN = 0, oF = 0, oH = 0, oW = 0;
+};
+
+static size_t esize_of(int dtype) { return dtype == PATDNN_F16 ? 2 : 4; }
+
+extern "C" {
+
+int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pattern_set, int32_t n_patterns,
+                  const patdnn_desc *desc, patdnn_handle *out) {
+    if (!weights || !mask || !pattern_set || !desc || !out) return PATDNN_E_NULL;
+    if (desc->F < 1 || desc->C < 1 || desc->N < 0 || desc->H < 1 || desc->W < 1) return PATDNN_E_SHAPE;
+    if (desc->H > 65535 || desc->W > 65535 || desc->N > 65535) return PATDNN_E_SHAPE;
+    if (desc->dtype != PATDNN_F32 && desc->dtype != PATDNN_F16) return PATDNN_E_DTYPE;
+    if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_TILED) return PATDNN_E_DTYPE;
+    if (desc->filter_order != 0 && desc->filter_order != 1) return PATDNN_E_ORDER;
+    if (desc->filter_order == 1 && !desc->order) return PATDNN_E_NULL;
+    patdnn_layer *h = new (std::nothrow) patdnn_layer();
+    if (!h) return PATDNN_E_ALLOC;
+    int rc = PATDNN_OK;
+    try {
+        rc = build_fkw(weights, mask, pattern_set, n_patterns, desc->F, desc->C, desc->dtype,
+                       desc->filter_order == 1 ? desc->order : nullptr, h->fkw);
+        if (rc == PATDNN_OK) {
+            h->desc = *desc;
+            h->desc.order = nullptr;
+            h->bias.assign(desc->F, 0.f);
+            if (desc->bias) std::memcpy(h->bias.data(), desc->bias, sizeof(float) * desc->F);
+            h->desc.bias = nullptr;
+            // resolve the variant
+            const bool can_tile = tiled_supported(h->fkw, desc->N, desc->H, desc->W, desc->dtype);
+            if (desc->variant == PATDNN_VARIANT_AUTO)
+                h->variant = can_tile ? PATDNN_VARIANT_TILED : PATDNN_VARIANT_REORDER;
+            else
+                h->variant = desc->variant;
+            if (h->variant == PATDNN_VARIANT_TILED && !can_tile) rc = PATDNN_E_SHAPE;
+        }
+        TiledLayout lay;
+        if (rc == PATDNN_OK && h->variant == PATDNN_VARIANT_TILED)
+            rc = plan_tiled(h->fkw, desc->N, desc->H, desc->W, desc->dtype, h->plan, lay);
+        if (rc == PATDNN_OK && !(desc->flags & PATDNN_FLAG_HOST_ONLY)) {
+            int dev = -1;
+            cudaError_t e = cudaGetDevice(&dev);
+            if (e != cudaSuccess) {
+                rc = cuda_fail(e, "cudaGetDevice");
+            } else {
+                h->device = dev;
+                const Fkw &k = h->fkw;
+                if (h->variant == PATDNN_VARIANT_TILED) {
+                    rc = upload(lay.desc, &h->d_desc, h->owned);
+                    if (!rc) rc = upload(lay.wts, &h->d_wts, h->owned);
+                    if (!rc) rc = upload(lay.seg, &h->d_seg, h->owned);
+                    if (!rc) rc = upload(lay.seglen, &h->d_seglen, h->owned);
+                    if (!rc) rc = upload(k.reorder, &h->d_reorder, h->owned);
+                    if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
+                    h->device_bytes = static_cast<int64_t>(lay.desc.size()) * 20 + lay.seg.size() * 8 + k.F * 8;
+                    if (!rc) {
+                        cudaError_t pe = prepare_tiled(h->plan, desc->dtype);
+                        if (pe != cudaSuccess) rc = cuda_fail(pe, "cudaFuncSetAttribute(shared memory)");
+                    }
+                } else {
+                    rc = upload(k.offset, &h->d_offset, h->owned);
+                    if (!rc) rc = upload(k.reorder, &h->d_reorder, h->owned);
+                    if (!rc) rc = upload(k.index, &h->d_index, h->owned);
+                    if (!rc) rc = upload(k.stride, &h->d_stride, h->owned);
+                    if (!rc) rc = upload(k.weight_f32, &h->d_weight, h->owned);
+                    if (!rc) rc = upload(k.patterns, &h->d_patterns, h->owned);
+                    if (!rc) rc = upload(k.kernel_pid, &h->d_kernel_pid, h->owned);
+                    if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
+                    h->device_bytes = static_cast<int64_t>(k.K) * 24 + k.F * (4 * (k.P + 1) + 12);
+                    if (!rc && h->variant == PATDNN_VARIANT_NOOPT) {
+                        std::vector<int32_t> slot(static_cast<size_t>(k.F) * k.C, -1);
+                        for (int i = 0; i < k.F; ++i)
+                            for (int32_t kk = k.offset[i]; kk < k.offset[i + 1]; ++kk)
+                                slot[static_cast<size_t>(k.reorder[i]) * k.C + k.index[kk]] = kk;
+                        rc = upload(slot, &h->d_dense_slot, h->owned);
+                        h->device_bytes += static_cast<int64_t>(slot.size()) * 4;
+                    }
+                }
+                if (!rc) h->on_device = true;
+            }
+        }
+    } catch (const std::bad_alloc &) {
+        rc = PATDNN_E_ALLOC;
+    }
+    if (rc != PATDNN_OK) {
+        patdnn_free(h);
+        return rc;
+    }
+    *out = h;
+    return PATDNN_OK;
+}
+
+int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
+    if (!h || !in || !out) return PATDNN_E_NULL;
+    if (!h->on_device) return PATDNN_E_NO_DEVICE;
+    const patdnn_desc &d = h->desc;
+    if (d.N == 0) return PATDNN_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (h->variant == PATDNN_VARIANT_TILED) {
+        TiledParams p{};
+        p.in = in; p.out = out;
+        p.desc = h->d_desc; p.wts = reinterpret_cast<const float4 *>(h->d_wts);
+        p.seg = h->d_seg; p.seglen = h->d_seglen; p.reorder = h->d_reorder; p.bias = h->d_bias;
+        p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
+        p.TXn = h->plan.TXn; p.TYn = h->plan.TYn; p.tiles_total = h->plan.tiles_total;
+        p.pitch = h->plan.pitch; p.lead = h->plan.lead; p.rows_max = h->plan.rows_max;
+        p.nchunk = h->plan.nchunk; p.CC = h->plan.cfg.CC; p.nblk = h->plan.nblk; p.seg_cap = h->plan.seg_cap;
+        p.copy_bytes = h->plan.copy_bytes; p.relu = d.relu;
+        e = launch_tiled(h->plan, p, d.dtype, st);
+    } else {
+        SimpleParams p{};
+        p.in = in; p.out = out;
+        p.offset = h->d_offset; p.reorder = h->d_reorder; p.index = h->d_index; p.stride = h->d_stride;
+        p.weight = reinterpret_cast<const float4 *>(h->d_weight); p.patterns = h->d_patterns;
+        p.kernel_pid = h->d_kernel_pid; p.dense_slot = h->d_dense_slot; p.bias = h->d_bias;
+        p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F; p.P = h->fkw.P; p.relu = d.relu;
+        e = launch_simple(p, h->variant, d.dtype, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PATDNN_OK;
+}
+
+int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void *stream) {
+    if (!h || !in_host || !out_host) return PATDNN_E_NULL;
+    if (!h->on_device) return PATDNN_E_NO_DEVICE;
+    const patdnn_desc &d = h->desc;
+    const size_t es = esize_of(d.dtype);
+    const size_t in_b = static_cast<size_t>(d.N) * d.C * d.H * d.W * es;
+    const size_t out_b = static_cast<size_t>(d.N) * d.F * d.H * d.W * es;
+    if (in_b == 0) return PATDNN_OK;
+    if (!h->d_in_stage) {
+        CU(cudaMalloc(&h->d_in_stage, in_b));
+        h->owned.push_back(h->d_in_stage);
+        CU(cudaMalloc(&h->d_out_stage, out_b));
+        h->owned.push_back(h->d_out_stage);
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpyAsync(h->d_in_stage, in_host, in_b, cudaMemcpyHostToDevice, st));
+    const int rc = patdnn_conv(h, h->d_in_stage, h->d_out_stage, stream);
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(out_host, h->d_out_stage, out_b, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return PATDNN_OK;
+}
+
+int patdnn_free(patdnn_handle h) {
+    if (!h) return PATDNN_OK;
+    for (void *p : h->owned) cudaFree(p);
+    delete h;
+    return PATDNN_OK;
+}
+
+int patdnn_export(patdnn_handle h, patdnn_fkw_view *v) {
+    if (!h || !v) return PATDNN_E_NULL;
+    const Fkw &k = h->fkw;
+    v->F = k.F; v->C = k.C; v->P = k.P; v->K = k.K;
+    v->offset = k.offset.data();
+    v->reorder = k.reorder.data();
+    v->index = k.index.data();
+    v->stride = k.stride.data();
+    v->weight = k.dtype == PATDNN_F16 ? static_cast<const void *>(k.weight_f16.data())
+                                      : static_cast<const void *>(k.weight_f32.data());
+    return PATDNN_OK;
+}
+
+int patdnn_decode(patdnn_handle h, float *dense_out) {
+    if (!h || !dense_out) return PATDNN_E_NULL;
+    decode_fkw(h->fkw, dense_out);
+    return PATDNN_OK;
+}
+
+int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
+    if (!h || !info) return PATDNN_E_NULL;
+    std::memset(info, 0, sizeof(*info));
+    info->variant = h->variant;
+    info->device_bytes = h->device_bytes;
+    if (h->variant == PATDNN_VARIANT_TILED) {
+        const TiledPlan &p = h->plan;
+        info->tile_rows = p.cfg.TY; info->tile_cols = kTileCols;
+        info->filters_per_warp = p.cfg.FR;
+        info->warps_per_cta = p.cfg.PW * p.cfg.FW;
+        info->channels_per_stage = p.cfg.CC;
+        info->channel_splits = 1;
+        info->grid_x = p.grid_pix * p.grid_fg; info->grid_y = 1; info->grid_z = 1;
+        info->smem_bytes = p.smem_bytes;
+        info->entries = p.entries;
+    } else {
+        info->tile_rows = 1; info->tile_cols = 1; info->filters_per_warp = 1; info->warps_per_cta = 8;
+        info->channels_per_stage = 0; info->channel_splits = 1;
+        info->grid_x = (h->desc.H * h->desc.W + 255) / 256; info->grid_y = h->desc.F; info->grid_z = h->desc.N;
+        info->entries = h->fkw.K;
+    }
+    return PATDNN_OK;
+}
+
+int patdnn_maxpool2x2(const void *in, void *out, int32_t N, int32_t C, int32_t H, int32_t W, int32_t dtype,
+                      void *stream) {
+    if (!in || !out) return PATDNN_E_NULL;
+    if (N < 0 || C < 1 || H < 2 || W < 2) return PATDNN_E_SHAPE;
+    if (dtype != PATDNN_F32 && dtype != PATDNN_F16) return PATDNN_E_DTYPE;
+    cudaError_t e = launch_maxpool2x2(in, out, N, C, H, W, dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "maxpool launch");
+    if (N > 0) g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PATDNN_OK;
+}
+
+int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after, int32_t n, patdnn_stack *out) {
+    if (!handles || !out) return PATDNN_E_NULL;
+    if (n < 1) return PATDNN_E_SHAPE;
+    patdnn_stack_s *s = new (std::nothrow) patdnn_stack_s();
+    if (!s) return PATDNN_E_ALLOC;
+    size_t max_bytes = 0;
+    int32_t N = 0, C = 0, H = 0, W = 0, dtype = 0;
+    for (int i = 0; i < n; ++i) {
+        patdnn_handle h = handles[i];
+        if (!h) { delete s; return PATDNN_E_NULL; }
+        if (!h->on_device) { delete s; return PATDNN_E_NO_DEVICE; }
+        const patdnn_desc &d = h->desc;
+        if (i == 0) { N = d.N; C = d.C; H = d.H; W = d.W; dtype = d.dtype; }
+        if (d.N != N || d.C != C || d.H != H || d.W != W || d.dtype != dtype) { delete s; return PATDNN_E_STACK; }
+        C = d.F;
+        max_bytes = std::max(max_bytes, static_cast<size_t>(N) * C * H * W * esize_of(dtype));
+        const int pool = pool_after ? pool_after[i] : 0;
+        if (pool) {
+            if (H < 2 || W < 2) { delete s; return PATDNN_E_STACK; }
+            H /= 2; W /= 2;
+        }
+        s->layers.push_back(h);
+        s->pool.push_back(pool);
+    }
+    s->oN = N; s->oF = C; s->oH = H; s->oW = W;
+    s->buf_bytes = std::max<size_t>(max_bytes, 16);
+    const patdnn_desc &d0 = handles[0]->desc;
+    s->in_bytes = static_cast<size_t>(d0.N) * d0.C * d0.H * d0.W * esize_of(dtype);
+    s->out_bytes = static_cast<size_t>(N) * C * H * W * esize_of(dtype);
+    for (int b = 0; b < 2; ++b) {
+        cudaError_t e = cudaMalloc(&s->buf[b], s->buf_bytes);
+        if (e != cudaSuccess) { patdnn_stack_free(s); return cuda_fail(e, "cudaMalloc(stack buffer)"); }
+    }
+    *out = s;
+    return PATDNN_OK;
+}
+
+int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
+    if (!s || !in || !out) return PATDNN_E_NULL;
+    const void *cur = in;
+    int which = 0;
+    const int n = static_cast<int>(s->layers.size());
+    for (int i = 0; i < n; ++i) {
+        patdnn_handle h = s->layers[i];
+        const patdnn_desc &d = h->desc;
+        const bool last = (i == n - 1);
+        void *dst = (last && !s->pool[i]) ? out : s->buf[which];
+        int rc = patdnn_conv(h, cur, dst, stream);
+        if (rc) return rc;
+        cur = dst;
+        which ^= 1;
+        if (s->pool[i]) {
+            void *pdst = last ? out : s->buf[which];
+            rc = patdnn_maxpool2x2(cur, pdst, d.N, d.F, d.H, d.W, d.dtype, stream);
+            if (rc) return rc;
+            cur = pdst;
+            which ^= 1;
+        }
+    }
+    return PATDNN_OK;
+}
+
+int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *out_host, void *stream) {
+    if (!s || !in_host || !out_host) return PATDNN_E_NULL;
+    if (!s->d_in) {
+        CU(cudaMalloc(&s->d_in, std::max<size_t>(s->in_bytes, 16)));
+        CU(cudaMalloc(&s->d_out, std::max<size_t>(s->out_bytes, 16)));
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpyAsync(s->d_in, in_host, s->in_bytes, cudaMemcpyHostToDevice, st));
+    const int rc = patdnn_stack_run(s, s->d_in, s->d_out, stream);
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(out_host, s->d_out, s->out_bytes, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return PATDNN_OK;
+}
+
+int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, int32_t *W) {
+    if (!s || !N || !F || !H || !W) return PATDNN_E_NULL;
+    *N = s->oN; *F = s->oF; *H = s->oH; *W = s->oW;
+    return PATDNN_OK;
+}
+
+int patdnn_stack_free(patdnn_stack s) {
+    if (!s) return PATDNN_OK;
+    for (int b = 0; b < 2; ++b)
+        if (s->buf[b]) cudaFree(s->buf[b]);
+    if (s->d_in) cudaFree(s->d_in);
+    if (s->d_out) cudaFree(s->d_out);
+    delete s;
+    return PATDNN_OK;
+}
+
+int64_t patdnn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+void patdnn_reset_launch_count(void) { g_launches.store(0, std::memory_order_relaxed); }
+
+const char *patdnn_strerror(int status) {
+    switch (status) {
+        case PATDNN_OK: return "ok";
+        case PATDNN_E_NULL: return "a required pointer is NULL";
+        case PATDNN_E_SHAPE: return "unsupported or inconsistent shape";
+        case PATDNN_E_PATTERN_SET: return "pattern set is not a list of distinct 4-of-9 patterns (1..32 entries)";
+        case PATDNN_E_MASK: return "a kernel mask is neither empty nor a pattern of the set";
+        case PATDNN_E_ORDER: return "filter order is not a permutation";
+        case PATDNN_E_CUDA: return "CUDA call failed";
+        case PATDNN_E_NO_DEVICE: return "handle has no device image (host-only encode or no CUDA device)";
+        case PATDNN_E_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case PATDNN_E_DTYPE: return "unknown dtype or variant";
+        case PATDNN_E_ALLOC: return "host allocation failed";
+        case PATDNN_E_STACK: return "stack layers do not chain";
+        default: return "unknown status";
+    }
+}
+
+const char *patdnn_last_cuda_error(void) { return g_cuda_error.c_str(); }
+const char *patdnn_version(void) { return "patdnn-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

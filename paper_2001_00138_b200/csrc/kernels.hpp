@@ -1,0 +1,94 @@
+// Internal interfaces between the C ABI, the host planners and the CUDA kernels.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <vector>
+
+#include "fkw_encoder.hpp"
+
+namespace patdnn {
+
+// ---- generic kernels (kernels_simple.cu) -------------------------------------------------------------------
+struct SimpleParams {
+    const void *in;
+    void *out;
+    const int32_t *offset;      // [F+1]
+    const int32_t *reorder;     // [F]
+    const int32_t *index;       // [K]
+    const int32_t *stride;      // [F][P+1]
+    const float4 *weight;       // [K] four kept weights (fp32 values; half-rounded for fp16 layers)
+    const uint16_t *patterns;   // [P]
+    const int32_t *kernel_pid;  // [K]
+    const int32_t *dense_slot;  // [F][C] stored kernel id of (original filter, channel) or -1 (no-opt variant only)
+    const float *bias;          // [F] original numbering
+    int N, C, H, W, F, P, relu;
+};
+
+cudaError_t launch_simple(const SimpleParams &p, int variant, int dtype, cudaStream_t stream);
+cudaError_t launch_maxpool2x2(const void *in, void *out, int N, int C, int H, int W, int dtype, cudaStream_t stream);
+
+// ---- tiled kernel (kernels_tiled.cu) -----------------------------------------------------------------------
+// Patterns the tiled kernel has straight-line code for.  A layer whose pattern set is a subset (in any order) runs
+// on the tiled kernel; any other set runs on the generic FKW kernel.
+constexpr int kBuiltinPatterns = 12;
+extern const uint16_t kBuiltinPatternMasks[kBuiltinPatterns];
+
+constexpr int kTileCols = 4;          // output columns per thread
+
+struct TiledConfig {
+    int TY;          // output rows per thread
+    int FR;          // filters register-blocked per warp
+    int PW;          // pixel warps per CTA (each covers 32 consecutive thread tiles)
+    int FW;          // filter warps per CTA (each covers FR consecutive filter positions)
+    int CC;          // input channels per shared-memory stage
+    int NS;          // stages
+};
+
+struct TiledPlan {
+    TiledConfig cfg{};
+    int TXn = 0, TYn = 0;       // thread tiles per image row / tile rows per image
+    int tiles_total = 0;        // N * TYn * TXn
+    int pitch = 0;              // shared-memory row pitch in elements
+    int lead = 0;               // zero elements in front of column 0 of every row
+    int rows_max = 0;           // rows staged per CTA
+    int nchunk = 0;             // ceil(C / CC)
+    int nblk = 0;               // filter blocks, ceil(F / FR)
+    int seg_cap = 0;            // largest (block, chunk) entry segment, entries (multiple of 4)
+    int copy_bytes = 0;         // bytes per asynchronous copy when staging rows: 16, 8 or 4
+    int grid_pix = 0, grid_fg = 0;
+    int smem_bytes = 0;
+    int64_t entries = 0;
+};
+
+struct TiledLayout {            // host image of the private device layout
+    std::vector<uint32_t> desc; // entry descriptors
+    std::vector<float> wts;     // 4 floats per entry
+    std::vector<int32_t> seg;   // [nblk*nchunk] start of each segment (entries)
+    std::vector<int32_t> seglen;// [nblk*nchunk] entries in the segment (multiple of 4, END included)
+};
+
+struct TiledParams {
+    const void *in;
+    void *out;
+    const uint32_t *desc;
+    const float4 *wts;
+    const int32_t *seg;
+    const int32_t *seglen;
+    const int32_t *reorder;
+    const float *bias;
+    int N, C, H, W, F;
+    int TXn, TYn, tiles_total;
+    int pitch, lead, rows_max;
+    int nchunk, CC, nblk, seg_cap, copy_bytes;
+    int relu;
+};
+
+// Can the tiled kernel run this layer (pattern set inside the builtin table, supported shape and dtype)?
+bool tiled_supported(const Fkw &fkw, int N, int H, int W, int dtype);
+// Pick a configuration for the shape and lay the kernels out for it.
+int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, TiledLayout &layout);
+cudaError_t launch_tiled(const TiledPlan &plan, const TiledParams &p, int dtype, cudaStream_t stream);
+cudaError_t prepare_tiled(const TiledPlan &plan, int dtype);   // opt in to the dynamic shared memory size
+
+}  // namespace patdnn

@@ -1,0 +1,184 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from paper_2001_00138_b200 import build, synth
+from util import TOL_F16, TOL_F32, assert_close, gpu_layer, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build_library()
+    from paper_2001_00138_b200 import binding
+    binding.load()
+    return binding
+
+
+VARIANTS = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3}
+
+
+@pytest.mark.parametrize("variant", ["tiled", "reorder", "noopt"])
+def test_config1(variant):
+    L = synth.config1()
+    got, plan = gpu_layer(L, variant=VARIANTS[variant])
+    assert plan["variant"] == VARIANTS[variant]
+    assert_close(got, oracle_layer(L), TOL_F32, f"config1/{variant}")
+
+
+# (N, C, F, H, W, n_patterns, prune): ragged tails in every dimension, widths that are not multiples of 4 or 2,
+# single rows/columns, batches that straddle a warp's tile range, more filters than one CTA holds.
+ODD_SHAPES = [
+    (2, 3, 5, 5, 5, 8, 0.0), (1, 4, 20, 7, 7, 8, 0.3), (3, 8, 33, 14, 14, 12, 0.5), (2, 16, 64, 9, 13, 8, 0.6),
+    (1, 5, 7, 1, 1, 4, 0.0), (1, 6, 40, 2, 30, 6, 0.2), (5, 9, 17, 3, 4, 8, 0.4), (2, 20, 130, 16, 16, 8, 0.7),
+    (1, 3, 16, 40, 36, 8, 0.0), (4, 12, 24, 6, 10, 12, 0.9), (1, 33, 70, 18, 66, 8, 0.5), (7, 2, 3, 4, 8, 8, 0.0),
+]
+
+
+@pytest.mark.parametrize("shape", ODD_SHAPES)
+@pytest.mark.parametrize("variant", ["tiled", "reorder"])
+def test_odd_shapes(shape, variant):
+    N, C, F, H, W, npat, prune = shape
+    L = synth.make_layer("odd", F=F, C=C, N=N, H=H, W=W, seed=hash(shape) % 10000, n_patterns=npat, prune=prune,
+                         bias_std=0.2, x_dist="normal", relu=(F % 2 == 1))
+    got, _ = gpu_layer(L, variant=VARIANTS[variant])
+    assert_close(got, oracle_layer(L), TOL_F32, f"{shape}/{variant}")
+
+
+def test_noopt_matches_on_pruned_layer():
+    L = synth.make_layer("n", F=24, C=18, N=2, H=11, W=9, seed=31, prune=0.5, bias_std=0.1)
+    got, _ = gpu_layer(L, variant=VARIANTS["noopt"])
+    assert_close(got, oracle_layer(L), TOL_F32, "noopt")
+
+
+def test_empty_filters_and_caller_order():
+    L = synth.make_layer("e", F=40, C=12, N=2, H=10, W=12, seed=77, prune=0.5, bias_std=0.5)
+    L.mask[3] = 0
+    L.mask[17] = 0
+    ref = oracle_layer(L)
+    for variant in ("tiled", "reorder"):
+        got, _ = gpu_layer(L, variant=VARIANTS[variant])
+        assert_close(got, ref, TOL_F32, variant)
+        assert np.all(got[:, 3] == max(L.bias[3], 0.0))
+        got, _ = gpu_layer(L, variant=VARIANTS[variant], order=synth.random_filter_order(40, 5))
+        assert_close(got, ref, TOL_F32, variant + "/random order")
+
+
+def test_output_is_fully_written_and_input_untouched():
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    L = synth.make_layer("w", F=19, C=7, N=3, H=13, W=10, seed=8, prune=0.4)
+    layer = B.encode(L.weights, L.mask, L.patterns, N=3, H=13, W=10, relu=True, bias=L.bias)
+    x = torch.from_numpy(L.x).cuda()
+    x0 = x.clone()
+    canary = torch.full((3 * 19 * 13 * 10 + 64,), -7.0, device="cuda")
+    out = canary[32:-32].view(3, 19, 13, 10)
+    layer.conv(x, out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert torch.equal(x, x0)
+    assert torch.all(canary[:32] == -7.0) and torch.all(canary[-32:] == -7.0)
+    assert torch.all(out >= 0)
+    layer.free()
+
+
+def test_config2_full_size():
+    L = synth.config2()
+    ref = oracle_layer(L)
+    got, plan = gpu_layer(L)
+    assert plan["variant"] == 3
+    assert_close(got, ref, TOL_F32, "config2")
+    got, _ = gpu_layer(L, via_host=True)
+    assert_close(got, ref, TOL_F32, "config2 via host buffers")
+
+
+@pytest.mark.parametrize("i", range(4))
+@pytest.mark.parametrize("N", [1, 3])
+def test_resnet_shapes_fp16(i, N):
+    L = synth.resnet50_layer(i, N=N)
+    ref = oracle_layer(L)
+    for variant in ("auto", "reorder"):
+        got, _ = gpu_layer(L, variant=VARIANTS[variant])
+        assert_close(got, ref, TOL_F16, f"resnet {i} N={N} {variant}")
+
+
+@pytest.mark.parametrize("npat,prune", [(4, 0.0), (6, 0.5), (8, 0.75), (12, 0.9)])
+def test_sweep_points_reduced_batch(npat, prune):
+    L = synth.sweep_layer(npat, prune, N=3)
+    ref = oracle_layer(L)
+    got, _ = gpu_layer(L)
+    assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune}")
+    got, _ = gpu_layer(L, order=synth.random_filter_order(512, 1))
+    assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune} random filter order")
+
+
+def test_vgg_stack_reduced_spatial_per_layer_and_chained():
+    """All 13 layers at 1/4 spatial size, batch 2: each GPU layer is fed the oracle's input for that layer
+    (binding check), and the chained GPU stack is compared with the chained oracle."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    scale, N = 4, 2
+    x = synth.vgg16_input(N, scale)
+    layers, handles = [], []
+    cur = x
+    for i in range(13):
+        L = synth.vgg16_layer(i, N=N, spatial_scale=scale)
+        ref = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+        got, _ = gpu_layer(L, x=cur)
+        assert_close(got, ref, TOL_F32, f"vgg layer {i + 1}")
+        cur = oracle.maxpool2x2(ref) if i in synth.VGG16_POOL_AFTER else ref
+        layers.append(L)
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, relu=True, bias=L.bias))
+    pools = [1 if i in synth.VGG16_POOL_AFTER else 0 for i in range(13)]
+    stack = B.Stack(handles, pools)
+    assert stack.out_shape() == cur.shape
+    xt = torch.from_numpy(x).cuda()
+    out = torch.empty(cur.shape, device="cuda")
+    stack.run(xt, out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert_close(out.cpu().numpy(), cur, 10 * TOL_F32, "vgg chained")      # 13 layers of rounding compound
+    out_h = np.empty(cur.shape, dtype=np.float32)
+    stack.run_host(x, out_h)
+    assert np.array_equal(out_h, out.cpu().numpy())
+    stack.free()
+    for h in handles:
+        h.free()
+
+
+@pytest.mark.parametrize("i,N", [(0, 32), (1, 32), (5, 32), (12, 32), (3, 1), (8, 1), (11, 1)])
+def test_vgg_full_size_sampled(i, N):
+    """Full-size layers in the benchmark's launch configuration; outputs sampled and checked one by one."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    L = synth.vgg16_layer(i, N=N)
+    rng = np.random.Generator(np.random.PCG64(900 + i))
+    x = rng.random((N, L.C, L.H, L.W), dtype=np.float32)
+    layer = B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, relu=True, bias=L.bias)
+    xt = torch.from_numpy(x).cuda()
+    out = torch.full((N, L.F, L.H, L.W), float("nan"), device="cuda")
+    layer.conv(xt, out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(out).all())
+    got = out.cpu().numpy()
+    pts = [(0, 0, 0, 0), (N - 1, L.F - 1, L.H - 1, L.W - 1), (N - 1, 0, 0, L.W - 1), (0, L.F - 1, L.H - 1, 0)]
+    for _ in range(300):
+        pts.append((int(rng.integers(N)), int(rng.integers(L.F)), int(rng.integers(L.H)), int(rng.integers(L.W))))
+    ref = np.asarray([oracle.conv3x3_point(x, L.weights, L.mask, L.bias, True, *p) for p in pts])
+    vals = np.asarray([got[p] for p in pts])
+    rms = float(np.sqrt(np.mean(got.astype(np.float64) ** 2)))
+    assert np.all(np.abs(vals - ref) <= TOL_F32 * np.maximum(np.abs(ref), rms)), f"vgg L{i + 1} N={N}"
+    layer.free()
+
+
+def test_maxpool_matches_oracle():
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    x = np.random.Generator(np.random.PCG64(6)).standard_normal((3, 5, 14, 10)).astype(np.float32)
+    xt = torch.from_numpy(x).cuda()
+    out = torch.empty((3, 5, 7, 5), device="cuda")
+    B.maxpool2x2(xt, out, 3, 5, 14, 10, B.F32, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), oracle.maxpool2x2(x))

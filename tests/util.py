@@ -1,0 +1,52 @@
+"""Shared helpers for the tests: tolerance rule and thin runners around the binding and the oracle."""
+import numpy as np
+
+TOL_F32 = 1e-4     # max relative error, fp32 storage
+TOL_F16 = 2e-3     # fp16 storage, fp32 accumulate
+
+
+def assert_close(got: np.ndarray, ref: np.ndarray, tol: float, what: str = "") -> float:
+    """|got - ref| <= tol * max(|ref|, rms(ref)) element by element; returns the worst ratio to that bound."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    rms = float(np.sqrt(np.mean(ref * ref))) if ref.size else 0.0
+    bound = tol * np.maximum(np.abs(ref), max(rms, 1e-30))
+    err = np.abs(got - ref)
+    worst = float((err / bound).max()) if ref.size else 0.0
+    if worst > 1.0:
+        i = np.unravel_index(np.argmax(err / bound), ref.shape)
+        raise AssertionError(f"{what}: |{got[i]} - {ref[i]}| exceeds {tol} * max(|ref|, rms={rms:.4g}) at {i} "
+                             f"(ratio {worst:.2f})")
+    return worst
+
+
+def oracle_layer(L, x=None):
+    import oracle
+    return oracle.conv3x3(L.x if x is None else x, L.weights, L.mask, L.bias, L.relu)
+
+
+def gpu_layer(L, x=None, variant=0, order=None, via_host=False):
+    """Encode L, run it on the GPU through the C ABI, return the output as float32 numpy."""
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    x = L.x if x is None else x
+    dt = B.F16 if L.dtype == "f16" else B.F32
+    tdt = torch.float16 if L.dtype == "f16" else torch.float32
+    N, C, H, W = x.shape
+    layer = B.encode(L.weights, L.mask, L.patterns, N=N, H=H, W=W, dtype=dt, relu=L.relu, bias=L.bias,
+                     order=order, variant=variant)
+    try:
+        if via_host:
+            xin = np.ascontiguousarray(x.astype(np.float16 if L.dtype == "f16" else np.float32))
+            out = np.empty((N, L.F, H, W), dtype=xin.dtype)
+            layer.conv_host(xin, out)
+            return out.astype(np.float32), layer.plan()
+        xt = torch.from_numpy(x).to("cuda", dtype=tdt).contiguous()
+        out = torch.full((N, L.F, H, W), float("nan"), device="cuda", dtype=tdt)
+        layer.conv(xt, out, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        return out.float().cpu().numpy(), layer.plan()
+    finally:
+        layer.free()
