@@ -302,7 +302,7 @@ template <int TY, int FR, int PW, int FW, int NS, typename T>
 cudaError_t launch_instance(const TiledPlan &plan, const TiledParams &p, cudaStream_t stream, bool prepare_only) {
     auto kern = conv_tiled_kernel<TY, FR, PW, FW, NS, T>;
     if (prepare_only)
-        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);  // per instance, not per layer
     const int grid = plan.grid_pix * plan.grid_fg;
     kern<<<grid, PW * FW * 32, plan.smem_bytes, stream>>>(p);
     return cudaGetLastError();

@@ -139,7 +139,8 @@ int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, 
     cfg.NS = 2;
     const int64_t tiles = static_cast<int64_t>(N) * ((H + cfg.TY - 1) / cfg.TY) * ((W + 3) / 4);
     if (tiles <= 32) cfg.PW = 1;
-    if ((fkw.F + cfg.FR - 1) / cfg.FR < cfg.FW) cfg.FW = std::max(1, (fkw.F + cfg.FR - 1) / cfg.FR);
+    const int nblk0 = (fkw.F + cfg.FR - 1) / cfg.FR;
+    cfg.FW = nblk0 >= 3 ? 4 : (nblk0 == 2 ? 2 : 1);
     const int kMaxSmem = 200 * 1024;
     for (int cc : {8, 4, 2, 1}) {
         cfg.CC = std::min(cc, fkw.C);
@@ -151,7 +152,7 @@ int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, 
     }
     build_layout(fkw, plan, layout, dtype);
     plan.smem_bytes = smem_bytes_for(plan, dtype);
-    if (plan.smem_bytes > 227 * 1024) return PATDNN_E_SHAPE;
+    if (plan.smem_bytes > 224 * 1024) return PATDNN_E_SHAPE;
     return PATDNN_OK;
 }
 
