@@ -8,8 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatdnn.so")
-SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "fkw_encoder.cpp", "tiled_plan.cpp"]
-HEADERS = ["kernels.hpp", "fkw_encoder.hpp", os.path.join("..", "..", "include", "patdnn.h")]
+SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "tiled_inst_4x8.cu",
+           "tiled_inst_4x4.cu", "tiled_inst_2x8.cu", "fkw_encoder.cpp", "tiled_plan.cpp"]
+HEADERS = ["kernels.hpp", "kernels_tiled.cuh", "fkw_encoder.hpp", os.path.join("generated", "tiled_cases.inc"),
+           os.path.join("..", "..", "include", "patdnn.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--threads", "0"]
 
@@ -31,6 +33,9 @@ def needs_build() -> bool:
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu/.cpp under csrc/ into one shared library; returns its path."""
+    sys.path.insert(0, CSRC)
+    import gen_cases                     # writes csrc/generated/tiled_cases.inc (the PTX FMA bodies)
+    gen_cases.generate()
     if not force and not needs_build():
         return LIB
     objs = []

@@ -59,8 +59,7 @@ struct patdnn_layer {
     uint16_t *d_patterns = nullptr;
     // tiled kernel
     TiledPlan plan;
-    uint32_t *d_desc = nullptr;
-    float *d_wts = nullptr;
+    uint32_t *d_rec = nullptr;
     int32_t *d_seg = nullptr, *d_seglen = nullptr;
     int64_t device_bytes = 0;
     // staging buffers of patdnn_conv_host
@@ -121,13 +120,12 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                 h->device = dev;
                 const Fkw &k = h->fkw;
                 if (h->variant == PATDNN_VARIANT_TILED) {
-                    rc = upload(lay.desc, &h->d_desc, h->owned);
-                    if (!rc) rc = upload(lay.wts, &h->d_wts, h->owned);
+                    rc = upload(lay.rec, &h->d_rec, h->owned);
                     if (!rc) rc = upload(lay.seg, &h->d_seg, h->owned);
                     if (!rc) rc = upload(lay.seglen, &h->d_seglen, h->owned);
                     if (!rc) rc = upload(k.reorder, &h->d_reorder, h->owned);
                     if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
-                    h->device_bytes = static_cast<int64_t>(lay.desc.size()) * 20 + lay.seg.size() * 8 + k.F * 8;
+                    h->device_bytes = static_cast<int64_t>(lay.rec.size()) * 4 + lay.seg.size() * 8 + k.F * 8;
                     if (!rc) {
                         cudaError_t pe = prepare_tiled(h->plan, desc->dtype);
                         if (pe != cudaSuccess) rc = cuda_fail(pe, "cudaFuncSetAttribute(shared memory)");
@@ -175,7 +173,7 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
     if (h->variant == PATDNN_VARIANT_TILED) {
         TiledParams p{};
         p.in = in; p.out = out;
-        p.desc = h->d_desc; p.wts = reinterpret_cast<const float4 *>(h->d_wts);
+        p.rec = h->d_rec;
         p.seg = h->d_seg; p.seglen = h->d_seglen; p.reorder = h->d_reorder; p.bias = h->d_bias;
         p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
         p.TXn = h->plan.TXn; p.TYn = h->plan.TYn; p.tiles_total = h->plan.tiles_total;

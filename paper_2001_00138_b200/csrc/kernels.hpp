@@ -42,7 +42,8 @@ struct TiledConfig {
     int PW;          // pixel warps per CTA (each covers 32 consecutive thread tiles)
     int FW;          // filter warps per CTA (each covers FR consecutive filter positions)
     int CC;          // input channels per shared-memory stage
-    int NS;          // stages
+    int NS;          // stages (2)
+    int MINB;        // CTAs per SM the instance is compiled for (register cap)
 };
 
 struct TiledPlan {
@@ -54,7 +55,7 @@ struct TiledPlan {
     int rows_max = 0;           // rows staged per CTA
     int nchunk = 0;             // ceil(C / CC)
     int nblk = 0;               // filter blocks, ceil(F / FR)
-    int seg_cap = 0;            // largest (block, chunk) entry segment, entries (multiple of 4)
+    int seg_cap = 0;            // largest (block, chunk) record segment, records
     int copy_bytes = 0;         // bytes per asynchronous copy when staging rows: 16, 8 or 4
     int grid_pix = 0, grid_fg = 0;
     int smem_bytes = 0;
@@ -62,17 +63,15 @@ struct TiledPlan {
 };
 
 struct TiledLayout {            // host image of the private device layout
-    std::vector<uint32_t> desc; // entry descriptors
-    std::vector<float> wts;     // 4 floats per entry
-    std::vector<int32_t> seg;   // [nblk*nchunk] start of each segment (entries)
-    std::vector<int32_t> seglen;// [nblk*nchunk] entries in the segment (multiple of 4, END included)
+    std::vector<uint32_t> rec;  // 8 words per record: {w0, w1, w2, w3 (float bits), descriptor, 0, 0, 0}
+    std::vector<int32_t> seg;   // [nblk*nchunk] first record of each segment
+    std::vector<int32_t> seglen;// [nblk*nchunk] records in the segment (END included)
 };
 
 struct TiledParams {
     const void *in;
     void *out;
-    const uint32_t *desc;
-    const float4 *wts;
+    const uint32_t *rec;
     const int32_t *seg;
     const int32_t *seglen;
     const int32_t *reorder;

@@ -4,15 +4,18 @@
 // Private layout.  Filters are taken in FKR order (Section 5.2) in blocks of FR consecutive positions, so the
 // filters one warp register-blocks have (nearly) equal length -- the load-balance use of the filter reorder -- and
 // input channels are taken in chunks of CC.  For every (filter block, channel chunk) there is one segment of 32-bit
-// descriptors plus four weights each, sorted by input channel:
+// records (descriptor plus four weights), sorted by input channel:
 //     LOAD(channel)                       fetch that channel's input patch into registers, once for all the
 //                                         block's kernels on the channel (filter-level load redundancy elimination,
 //                                         Section 5.4)
 //     FMA(slot j, pattern p), w0..w3      accumulate kernel (filter slot j, this channel) with the straight-line
 //                                         code of pattern p (kernel-level elimination: the patch registers are
 //                                         reused by the four taps)
-//     END                                 (segments are padded with END to a multiple of four entries)
+//     END
+// Each record is 32 bytes: {w0, w1, w2, w3, descriptor, 0, 0, 0}.
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "../../include/patdnn.h"
@@ -76,8 +79,9 @@ static void fill_geometry(TiledPlan &pl, const Fkw &fkw, int N, int H, int W, in
 static int smem_bytes_for(const TiledPlan &pl, int dtype) {
     const int esize = dtype == PATDNN_F16 ? 2 : 4;
     const int in_stage = pl.cfg.CC * pl.rows_max * pl.pitch * esize + 16;
-    const int seg_stage = pl.cfg.FW * pl.seg_cap * 20;
-    return pl.cfg.NS * (in_stage + seg_stage);
+    const int seg_stage = pl.cfg.FW * pl.seg_cap * 32 + 32;
+    const int items = pl.rows_max * (pl.pitch * esize / pl.copy_bytes) * 8;     // per-CTA copy plan
+    return pl.cfg.NS * (in_stage + seg_stage) + items;
 }
 
 static void build_layout(const Fkw &fkw, TiledPlan &pl, TiledLayout &lay, int dtype) {
@@ -98,42 +102,50 @@ static void build_layout(const Fkw &fkw, TiledPlan &pl, TiledLayout &lay, int dt
     const uint32_t code_load = static_cast<uint32_t>(c.FR * kBuiltinPatterns);
     const uint32_t code_end = code_load + 1;
     const uint32_t ch_stride_bytes = static_cast<uint32_t>(pl.rows_max) * pl.pitch * esize;
-    lay.desc.clear(); lay.wts.clear();
+    lay.rec.clear();
     lay.seg.assign(nseg, 0); lay.seglen.assign(nseg, 0);
     int cap = 0;
+    auto push = [&](uint32_t desc, const float *w) {
+        uint32_t r[8] = {0, 0, 0, 0, desc, 0, 0, 0};
+        if (w) std::memcpy(r, w, 16);
+        lay.rec.insert(lay.rec.end(), r, r + 8);
+    };
     for (int s = 0; s < nseg; ++s) {
         std::vector<E> &v = bucket[s];
         std::sort(v.begin(), v.end(), [](const E &a, const E &b) { return a.cc != b.cc ? a.cc < b.cc : a.j < b.j; });
-        const size_t start = lay.desc.size();
+        const size_t start = lay.rec.size() / 8;
         lay.seg[s] = static_cast<int32_t>(start);
         int cur = -1;
         for (const E &e : v) {
             if (e.cc != cur) {
                 cur = e.cc;
-                lay.desc.push_back(code_load | ((static_cast<uint32_t>(cur) * ch_stride_bytes) << 10));
-                lay.wts.insert(lay.wts.end(), 4, 0.f);
+                push(code_load | ((static_cast<uint32_t>(cur) * ch_stride_bytes) << 10), nullptr);
             }
-            lay.desc.push_back(static_cast<uint32_t>(e.j * kBuiltinPatterns + e.pid));
-            const float *w = &fkw.weight_f32[static_cast<size_t>(e.k) * 4];
-            lay.wts.insert(lay.wts.end(), w, w + 4);
+            push(static_cast<uint32_t>(e.j * kBuiltinPatterns + e.pid), &fkw.weight_f32[static_cast<size_t>(e.k) * 4]);
         }
-        do {
-            lay.desc.push_back(code_end);
-            lay.wts.insert(lay.wts.end(), 4, 0.f);
-        } while ((lay.desc.size() - start) % 4 != 0);
-        lay.seglen[s] = static_cast<int32_t>(lay.desc.size() - start);
+        push(code_end, nullptr);
+        lay.seglen[s] = static_cast<int32_t>(lay.rec.size() / 8 - start);
         cap = std::max(cap, lay.seglen[s]);
     }
     pl.seg_cap = cap;
-    pl.entries = static_cast<int64_t>(lay.desc.size());
+    pl.entries = static_cast<int64_t>(lay.rec.size() / 8);
 }
 
 int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, TiledLayout &layout) {
     if (!tiled_supported(fkw, N, H, W, dtype)) return PATDNN_E_SHAPE;
-    // Blocking choice.  Every configuration keeps 128 fp32 accumulators per thread (FR filters x TY x 4 pixels).
+    // Blocking choice: (rows per thread, filters per warp).  The override is for tuning runs and tests.
     TiledConfig cfg{};
-    cfg.TY = (H % 4 == 0 && H >= 16) ? 4 : 2;
-    cfg.FR = 128 / (cfg.TY * kTileCols);
+    int ty = 4, fr = 4;
+    if (H < 4 || (H % 4 != 0 && H < 16)) { ty = 2; fr = 8; }
+    if (const char *ov = std::getenv("PATDNN_TILE")) {        // "TYxFR", e.g. 4x4
+        int a = 0, b = 0;
+        if (std::sscanf(ov, "%dx%d", &a, &b) == 2 &&
+            ((a == 4 && b == 8) || (a == 4 && b == 4) || (a == 2 && b == 8))) {
+            ty = a; fr = b;
+        }
+    }
+    cfg.TY = ty; cfg.FR = fr;
+    cfg.MINB = (ty * fr * 4 <= 64) ? 2 : 1;
     cfg.PW = 2;
     cfg.FW = 4;
     cfg.NS = 2;
@@ -141,13 +153,13 @@ int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, 
     if (tiles <= 32) cfg.PW = 1;
     const int nblk0 = (fkw.F + cfg.FR - 1) / cfg.FR;
     cfg.FW = nblk0 >= 3 ? 4 : (nblk0 == 2 ? 2 : 1);
-    const int kMaxSmem = 200 * 1024;
+    const int kMaxSmem = (cfg.MINB == 2 ? 100 : 200) * 1024;
     for (int cc : {8, 4, 2, 1}) {
         cfg.CC = std::min(cc, fkw.C);
         plan = TiledPlan();
         plan.cfg = cfg;
         fill_geometry(plan, fkw, N, H, W, dtype);
-        plan.seg_cap = ((cfg.FR + 1) * cfg.CC + 4) / 4 * 4;          // upper bound before the layout exists
+        plan.seg_cap = (cfg.FR + 1) * cfg.CC + 1;                    // upper bound before the layout exists
         if (smem_bytes_for(plan, dtype) <= kMaxSmem || cc == 1) break;
     }
     build_layout(fkw, plan, layout, dtype);
