@@ -141,7 +141,7 @@ def test_host_only_handle_refuses_to_run(B):
     assert e.value.status == 7
     info = layer.plan()
     assert info["variant"] == B.VARIANT_TILED and info["tile_cols"] == 4
-    assert info["filters_per_warp"] * info["tile_rows"] * info["tile_cols"] == 128
+    assert info["filters_per_warp"] * info["tile_rows"] * info["tile_cols"] in (64, 128)   # fp32 accumulators per thread
     assert info["entries"] >= 512 and info["smem_bytes"] <= 227 * 1024
     layer.free()
 
