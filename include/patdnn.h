@@ -60,7 +60,9 @@ enum {
     PATDNN_VARIANT_AUTO = 0,
     PATDNN_VARIANT_NOOPT = 1,     /* original filter order, per-kernel branch on the pattern, global loads */
     PATDNN_VARIANT_REORDER = 2,   /* walks the FKW arrays in pattern order (branch-free per run), global loads */
-    PATDNN_VARIANT_TILED = 3      /* shared-memory tile + halo, register patch reuse across taps and filters */
+    PATDNN_VARIANT_TILED = 3,     /* shared-memory tile + halo, register patch reuse across taps and filters */
+    PATDNN_VARIANT_DENSE_TC = 4   /* per-tap dense implicit GEMM on the tensor cores (tcgen05); fp32 layers use three
+                                     bf16 products of operands split into hi + lo; chosen where it beats TILED */
 };
 
 enum { PATDNN_FLAG_HOST_ONLY = 1 };   /* encode on the host only: no device is touched, patdnn_conv is refused */
@@ -111,6 +113,12 @@ PATDNN_API int patdnn_conv(patdnn_handle h, const void *in, void *out, void *str
  * live until patdnn_free.
  */
 PATDNN_API int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void *stream);
+
+/*
+ * patdnn_check -- wait for the device and report whether any kernel launched for this handle gave up on a bounded
+ * device-side wait (PATDNN_E_DEVICE_TIMEOUT) or a CUDA error is pending (PATDNN_E_CUDA).  Synchronous.
+ */
+PATDNN_API int patdnn_check(patdnn_handle h);
 
 /* patdnn_free -- release the handle and everything it owns (device and host).  NULL is accepted. */
 PATDNN_API int patdnn_free(patdnn_handle h);

@@ -17,13 +17,13 @@ LIB_PATH = os.path.join(HERE, "libpatdnn.so")
 
 OK = 0
 F32, F16 = 0, 1
-VARIANT_AUTO, VARIANT_NOOPT, VARIANT_REORDER, VARIANT_TILED = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_NOOPT, VARIANT_REORDER, VARIANT_TILED, VARIANT_DENSE_TC = 0, 1, 2, 3, 4
 FLAG_HOST_ONLY = 1
 STATUS_NAMES = {0: "OK", 1: "E_NULL", 2: "E_SHAPE", 3: "E_PATTERN_SET", 4: "E_MASK", 5: "E_ORDER", 6: "E_CUDA",
                 7: "E_NO_DEVICE", 8: "E_DEVICE_TIMEOUT", 9: "E_DTYPE", 10: "E_ALLOC", 11: "E_STACK"}
 
 EXPORTED_SYMBOLS = (
-    "patdnn_encode", "patdnn_conv", "patdnn_conv_host", "patdnn_free", "patdnn_export", "patdnn_decode",
+    "patdnn_encode", "patdnn_conv", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
     "patdnn_stack_free", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
     "patdnn_last_cuda_error", "patdnn_version",
@@ -76,6 +76,7 @@ def load() -> ctypes.CDLL:
     lib.patdnn_conv.argtypes = [vp, vp, vp, vp]
     lib.patdnn_conv_host.argtypes = [vp, vp, vp, vp]
     lib.patdnn_free.argtypes = [vp]
+    lib.patdnn_check.argtypes = [vp]
     lib.patdnn_export.argtypes = [vp, ctypes.POINTER(_FkwView)]
     lib.patdnn_decode.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.patdnn_plan.argtypes = [vp, ctypes.POINTER(_PlanInfo)]
@@ -128,6 +129,10 @@ class Layer:
         """patdnn_conv_host: host buffers in, host buffers out (copies inside the call)."""
         assert x.flags.c_contiguous and out.flags.c_contiguous
         _check(load().patdnn_conv_host(self._h, x.ctypes.data, out.ctypes.data, stream), "patdnn_conv_host")
+
+    def check(self) -> None:
+        """patdnn_check: synchronise and raise if a device-side bounded wait expired."""
+        _check(load().patdnn_check(self._h), "patdnn_check")
 
     def export(self) -> Dict[str, np.ndarray]:
         v = _FkwView()

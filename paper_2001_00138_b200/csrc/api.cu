@@ -1,6 +1,7 @@
 // C ABI of the library (declared in include/patdnn.h): handles, uploads, launches.  No torch types anywhere.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -62,6 +63,11 @@ struct patdnn_layer {
     uint32_t *d_rec = nullptr;
     int32_t *d_seg = nullptr, *d_seglen = nullptr;
     int64_t device_bytes = 0;
+    // dense tensor-core path
+    DensePlan dense;
+    uint16_t *d_wdense = nullptr;
+    void *d_act = nullptr;
+    int *d_status = nullptr;
     // staging buffers of patdnn_conv_host
     void *d_in_stage = nullptr, *d_out_stage = nullptr;
 };
@@ -85,7 +91,7 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
     if (desc->F < 1 || desc->C < 1 || desc->N < 0 || desc->H < 1 || desc->W < 1) return PATDNN_E_SHAPE;
     if (desc->H > 65535 || desc->W > 65535 || desc->N > 65535) return PATDNN_E_SHAPE;
     if (desc->dtype != PATDNN_F32 && desc->dtype != PATDNN_F16) return PATDNN_E_DTYPE;
-    if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_TILED) return PATDNN_E_DTYPE;
+    if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_DENSE_TC) return PATDNN_E_DTYPE;
     if (desc->filter_order != 0 && desc->filter_order != 1) return PATDNN_E_ORDER;
     if (desc->filter_order == 1 && !desc->order) return PATDNN_E_NULL;
     patdnn_layer *h = new (std::nothrow) patdnn_layer();
@@ -102,10 +108,26 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
             h->desc.bias = nullptr;
             // resolve the variant
             const bool can_tile = tiled_supported(h->fkw, desc->N, desc->H, desc->W, desc->dtype);
-            if (desc->variant == PATDNN_VARIANT_AUTO)
+            if (desc->variant == PATDNN_VARIANT_AUTO) {
                 h->variant = can_tile ? PATDNN_VARIANT_TILED : PATDNN_VARIANT_REORDER;
-            else
+                // Tensor cores only where the dense reformulation is expected to win: compare a time estimate of the
+                // zero-padded per-tap GEMMs with the CUDA-core kernel's rate on the kept weights (both measured on
+                // B200: ~900 TFLOP/s sustained for the 16-bit MMAs of this kernel, ~12 TFLOP/s for the tiled kernel).
+                if (!(desc->flags & PATDNN_FLAG_HOST_ONLY) && desc->N > 0 &&
+                    dense_supported(desc->F, desc->C, desc->N, desc->H, desc->W)) {
+                    DensePlan dp;
+                    plan_dense(desc->F, desc->C, desc->N, desc->H, desc->W, desc->dtype, dp);
+                    const double terms = desc->dtype == PATDNN_F16 ? 1.0 : 3.0;
+                    const double rows = static_cast<double>(dp.tiles_x) * dp.tiles_y * dp.tiles_n * 128.0;
+                    const double t_dense = terms * 2.0 * 9.0 * dp.Cp * dp.Fp * rows / 9.0e14 +
+                                           static_cast<double>(desc->N) * desc->H * desc->W * (desc->C * 4.0 + dp.Cp * 2.0 * dp.S) / 4.0e12 +
+                                           4e-6;
+                    const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / 1.2e13 + 4e-6;
+                    if (t_dense < t_tiled) h->variant = PATDNN_VARIANT_DENSE_TC;
+                }
+            } else {
                 h->variant = desc->variant;
+            }
             if (h->variant == PATDNN_VARIANT_TILED && !can_tile) rc = PATDNN_E_SHAPE;
         }
         TiledLayout lay;
@@ -119,7 +141,34 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
             } else {
                 h->device = dev;
                 const Fkw &k = h->fkw;
-                if (h->variant == PATDNN_VARIANT_TILED) {
+                if (h->variant == PATDNN_VARIANT_DENSE_TC) {
+                    if (!dense_supported(k.F, k.C, desc->N, desc->H, desc->W)) rc = PATDNN_E_SHAPE;
+                    if (!rc) {
+                        plan_dense(k.F, k.C, std::max(desc->N, 1), desc->H, desc->W, desc->dtype, h->dense);
+                        std::vector<uint16_t> wd;
+                        build_dense_weights(k, h->dense, wd);
+                        rc = upload(wd, &h->d_wdense, h->owned);
+                        h->device_bytes = static_cast<int64_t>(wd.size()) * 2;
+                    }
+                    if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
+                    if (!rc) {
+                        const size_t act_bytes = static_cast<size_t>(h->dense.S) * std::max(desc->N, 1) * desc->H *
+                                                 desc->W * h->dense.Cp * 2;
+                        cudaError_t ce = cudaMalloc(&h->d_act, act_bytes);
+                        if (ce != cudaSuccess) rc = cuda_fail(ce, "cudaMalloc(split activations)");
+                        else h->owned.push_back(h->d_act);
+                    }
+                    if (!rc) {
+                        std::vector<int> zero(4, 0);
+                        rc = upload(zero, &h->d_status, h->owned);
+                    }
+                    if (!rc) rc = make_dense_maps(h->dense, h->d_act, h->d_wdense, std::max(desc->N, 1), desc->H, desc->W, desc->dtype);
+                    if (rc == PATDNN_E_CUDA && g_cuda_error.empty()) g_cuda_error = "cuTensorMapEncodeTiled failed";
+                    if (!rc) {
+                        cudaError_t pe = prepare_dense(h->dense, desc->dtype);
+                        if (pe != cudaSuccess) rc = cuda_fail(pe, "cudaFuncSetAttribute(dense kernel)");
+                    }
+                } else if (h->variant == PATDNN_VARIANT_TILED) {
                     rc = upload(lay.rec, &h->d_rec, h->owned);
                     if (!rc) rc = upload(lay.seg, &h->d_seg, h->owned);
                     if (!rc) rc = upload(lay.seglen, &h->d_seglen, h->owned);
@@ -170,7 +219,16 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
     if (d.N == 0) return PATDNN_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if (h->variant == PATDNN_VARIANT_TILED) {
+    if (h->variant == PATDNN_VARIANT_DENSE_TC) {
+        DenseParams p{};
+        const DensePlan &pl = h->dense;
+        p.out = out; p.bias = h->d_bias; p.status = h->d_status;
+        p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
+        p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y;
+        p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
+        e = launch_dense(pl, p, in, h->d_act, d.dtype, st);
+        if (e == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);   // the layout kernel
+    } else if (h->variant == PATDNN_VARIANT_TILED) {
         TiledParams p{};
         p.in = in; p.out = out;
         p.rec = h->d_rec;
@@ -218,6 +276,21 @@ int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void 
     return PATDNN_OK;
 }
 
+int patdnn_check(patdnn_handle h) {
+    if (!h) return PATDNN_E_NULL;
+    if (!h->on_device) return PATDNN_E_NO_DEVICE;
+    CU(cudaDeviceSynchronize());
+    if (h->d_status) {
+        int st = 0;
+        CU(cudaMemcpy(&st, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+        if (st != 0) {
+            cudaMemset(h->d_status, 0, sizeof(int));
+            return PATDNN_E_DEVICE_TIMEOUT;
+        }
+    }
+    return PATDNN_OK;
+}
+
 int patdnn_free(patdnn_handle h) {
     if (!h) return PATDNN_OK;
     for (void *p : h->owned) cudaFree(p);
@@ -259,6 +332,12 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->grid_x = p.grid_pix * p.grid_fg; info->grid_y = 1; info->grid_z = 1;
         info->smem_bytes = p.smem_bytes;
         info->entries = p.entries;
+    } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
+        const DensePlan &p = h->dense;
+        info->tile_rows = p.TH; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
+        info->channels_per_stage = 64; info->channel_splits = 1;
+        info->grid_x = p.grid; info->grid_y = 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
+        info->entries = static_cast<int64_t>(9) * p.Fp * p.Cp;
     } else {
         info->tile_rows = 1; info->tile_cols = 1; info->filters_per_warp = 1; info->warps_per_cta = 8;
         info->channels_per_stage = 0; info->channel_splits = 1;

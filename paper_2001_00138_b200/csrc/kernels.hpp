@@ -1,5 +1,6 @@
 // Internal interfaces between the C ABI, the host planners and the CUDA kernels.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -89,5 +90,32 @@ bool tiled_supported(const Fkw &fkw, int N, int H, int W, int dtype);
 int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, TiledLayout &layout);
 cudaError_t launch_tiled(const TiledPlan &plan, const TiledParams &p, int dtype, cudaStream_t stream);
 cudaError_t prepare_tiled(const TiledPlan &plan, int dtype);   // opt in to the dynamic shared memory size
+
+// ---- dense tensor-core reformulation (umma_conv.cu) -----------------------------------------------------------
+struct DensePlan {
+    int S = 0;                  // operand planes: 2 (bf16 hi + lo, fp32 layers) or 1 (fp16 layers)
+    int Cp = 0, KB = 0;         // channels padded to a multiple of 64; channel blocks
+    int BN = 0, Fp = 0, n_ftiles = 0;
+    int TW = 0, TH = 0, TN = 0; // pixel box (columns, rows, images), TW*TH*TN <= 128
+    int tiles_x = 0, tiles_y = 0, tiles_n = 0;
+    int box_bytes = 0, stages = 0, smem_bytes = 0, grid = 0;
+    CUtensorMap mapA{}, mapB{};
+};
+
+struct DenseParams {
+    void *out;
+    const float *bias;
+    int *status;                // device word: 0 = ok, else the role whose bounded wait expired
+    int N, C, H, W, F;
+    int TW, TH, TN, tiles_x, tiles_y, n_ftiles;
+    int KB, stages, box_bytes, relu;
+};
+
+bool dense_supported(int F, int C, int N, int H, int W);
+void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl);
+void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16_t> &w);
+int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, int dtype);
+cudaError_t prepare_dense(const DensePlan &pl, int dtype);
+cudaError_t launch_dense(const DensePlan &pl, const DenseParams &p, const void *in, void *act, int dtype, cudaStream_t st);
 
 }  // namespace patdnn

@@ -1,0 +1,430 @@
+// Dense tensor-core reformulation of the pattern-sparse convolution for sm_100a (tcgen05 + TMEM + TMA).
+//
+// The layer is out = act(bias + sum_{tap} X_tap * W_tap): nine shifted views X_tap of the input times nine F x C
+// weight slices W_tap in which the pruned taps and kernels are zero.  As an implicit GEMM per tap this is a plain
+// dense contraction (M = pixels, N = filters, K = channels), which the 5th-generation tensor cores run far above the
+// FP32 FMA rate -- enough to pay for the zeros when the layer is not too sparse.  The planner uses this path only
+// where it beats the CUDA-core kernel.
+//
+// Precision.  fp32 layers must stay within 1e-4 of the fp64 oracle, which a single bf16/tf32 product cannot give.
+// Every fp32 operand is split x = hi + lo with hi = bf16(x), lo = bf16(x - hi) (16 significand bits together) and the
+// product is taken as hi*hi + hi*lo + lo*hi, three bf16 MMAs into one fp32 TMEM accumulator; the dropped lo*lo term
+// and the split rounding are below 2^-16 relative.  fp16 layers (2e-3) use one fp16 MMA on the stored values.
+//
+// Data flow.
+//   prep_act_kernel  : NCHW activations -> [S][N][H][W][Cp] (channels innermost, padded to a multiple of 64 with
+//                      zeros; S = 2 planes hi/lo for fp32 layers, 1 for fp16 layers);
+//   encode (host)    : weights -> [S][9][Fp][Cp] in the same split, zeros where pruned;
+//   conv_umma_kernel : one CTA = 128 output pixels (a TW x TH x TN box of the image batch) x BN filters.
+//       warp 0   TMA producer: per (channel block of 64, tap) loads the shifted pixel box (zero fill outside the image
+//                gives the padding) and the weight tile, 128-byte swizzle, multi-stage mbarrier ring;
+//       warp 1   one thread issues tcgen05.mma (M=128, N=BN, K=16) x 4 k-steps x 3 split terms per stage, accumulating
+//                in TMEM, and releases the stage with tcgen05.commit;
+//       warps 2-5 epilogue: tcgen05.ld the accumulator, bias + ReLU, store NCHW.
+// Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves through the normal exit
+// (TMEM is always deallocated).  No cluster multicast anywhere.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+
+#include "../../include/patdnn.h"
+#include "kernels.hpp"
+
+namespace patdnn {
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTileM = 128;
+constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
+constexpr uint32_t kSpinLimit = 1u << 21;    // bounded mbarrier polling: each poll may block up to ~1 us (hint below)
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait: returns false (and leaves *status set) when the phase did not complete within the polling budget.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *status, int code) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred P1;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2, 0x400;\n\t"
+            "selp.b32 %0, 1, 0, P1;\n\t}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if (*reinterpret_cast<volatile int *>(status) != 0) return false;      // another role already gave up
+    }
+    atomicCAS(status, 0, code);
+    return false;
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled shared-memory matrix descriptor: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);            // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                            // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                    // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                            // descriptor version for sm_100
+    d |= static_cast<uint64_t>(2) << 61;                            // layout: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: fp32 accumulate, A and B both K-major in the same 16-bit format (0 = f16, 1 = bf16).
+__host__ __device__ constexpr uint32_t instr_desc(int fmt, int n) {
+    return (1u << 4) | (static_cast<uint32_t>(fmt) << 7) | (static_cast<uint32_t>(fmt) << 10) |
+           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(addr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- activation layout change + operand split ---------------------------------------------------------------------
+// grid = (ceil(W/32), H, N), block = (32, 8).  One block moves a 32-pixel row segment for all channels.
+template <typename T>
+__global__ void __launch_bounds__(256) prep_act_kernel(const T *__restrict__ in, uint16_t *__restrict__ out, int N, int C,
+                                                       int H, int W, int Cp, int S) {
+    __shared__ float tile[64][33];
+    const int x0 = blockIdx.x * 32, y = blockIdx.y, n = blockIdx.z;
+    const int tx = threadIdx.x, tyq = threadIdx.y;
+    const size_t plane_out = static_cast<size_t>(N) * H * W * Cp;
+    for (int c0 = 0; c0 < Cp; c0 += 64) {
+        for (int cc = tyq; cc < 64; cc += 8) {
+            const int c = c0 + cc, x = x0 + tx;
+            float v = 0.f;
+            if (c < C && x < W) {
+                const T raw = in[((static_cast<size_t>(n) * C + c) * H + y) * W + x];
+                if constexpr (sizeof(T) == 2) v = __half2float(raw); else v = raw;
+            }
+            tile[cc][tx] = v;
+        }
+        __syncthreads();
+        // write: 32 pixels x 64 channels; a warp writes one pixel's 64 channels as 32 x (2 channels)
+        for (int px = tyq; px < 32; px += 8) {
+            const int x = x0 + px;
+            if (x < W) {
+                const float a = tile[2 * tx][px], b = tile[2 * tx + 1][px];
+                const size_t o = ((static_cast<size_t>(n) * H + y) * W + x) * Cp + c0 + 2 * tx;
+                if (S == 2) {
+                    const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+                    const __nv_bfloat16 al = __float2bfloat16_rn(a - __bfloat162float(ah));
+                    const __nv_bfloat16 bl = __float2bfloat16_rn(b - __bfloat162float(bh));
+                    const uint32_t hi = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) |
+                                        (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
+                    const uint32_t lo = static_cast<uint32_t>(__bfloat16_as_ushort(al)) |
+                                        (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
+                    *reinterpret_cast<uint32_t *>(out + o) = hi;
+                    *reinterpret_cast<uint32_t *>(out + plane_out + o) = lo;
+                } else {
+                    const uint32_t v = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(a))) |
+                                       (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(b))) << 16);
+                    *reinterpret_cast<uint32_t *>(out + o) = v;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---- the implicit-GEMM kernel -------------------------------------------------------------------------------------
+template <int BN, int TERMS, typename T>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
+    constexpr int S = (TERMS == 3) ? 2 : 1;                     // operand planes (hi, lo)
+    constexpr int A_BYTES = kTileM * 128;
+    constexpr int B_BYTES = BN * 128;
+    constexpr int STAGE_BYTES = S * (A_BYTES + B_BYTES);
+    constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) uint64_t bars[2 * 8 + 1];          // full[stages], empty[stages], accumulator ready
+    __shared__ uint32_t tmem_slot;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int stages = p.stages;
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[8]), bar_acc = smem_u32(&bars[16]);
+    int *status = p.status;
+
+    // tile coordinates: filter tile fastest so that CTAs sharing a pixel box run together (L2 reuse of the box)
+    const int ft = blockIdx.x % p.n_ftiles;
+    int pt = blockIdx.x / p.n_ftiles;
+    const int tix = pt % p.tiles_x; pt /= p.tiles_x;
+    const int tiy = pt % p.tiles_y; pt /= p.tiles_y;
+    const int x0 = tix * p.TW, y0 = tiy * p.TH, n0 = pt * p.TN, f0 = ft * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {   // TMEM allocation by one full warp; the same warp frees it at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    const int iters = 9 * p.KB;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t tx_bytes = S * (p.box_bytes + B_BYTES);
+            for (int it = 0; it < iters; ++it) {
+                const int s = it % stages, use = it / stages;
+                if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1, status, 1)) break;
+                const int cb = it / 9, tap = it - cb * 9;
+                const int r = tap / 3, sx = tap - 3 * r;
+                const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
+                mbar_expect_tx(bar_full + 8 * s, tx_bytes);
+#pragma unroll
+                for (int sp = 0; sp < S; ++sp) {
+                    tma_load_5d(base + sp * A_BYTES, &mapA, bar_full + 8 * s, cb * kKBlock, x0 + sx - 1, y0 + r - 1, n0, sp);
+                    tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * s, cb * kKBlock, f0, tap, sp);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % stages, use = it / stages;
+                ok = mbar_wait(bar_full + 8 * s, use & 1, status, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
+                const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + A_BYTES);
+                const uint64_t b_hi = smem_desc_sw128(base + S * A_BYTES), b_lo = smem_desc_sw128(base + S * A_BYTES + B_BYTES);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {                   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes
+                    const uint64_t koff = static_cast<uint64_t>(2 * k);
+                    umma_f16(tmem_base, a_hi + koff, b_hi + koff, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    if constexpr (TERMS == 3) {
+                        umma_f16(tmem_base, a_hi + koff, b_lo + koff, idesc, 1u);
+                        umma_f16(tmem_base, a_lo + koff, b_hi + koff, idesc, 1u);
+                    }
+                }
+                umma_commit(bar_empty + 8 * s);                 // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(bar_acc);
+        }
+    } else {
+        // epilogue: warp w reads TMEM lanes 32*(w%4) .. +31; lane = output pixel of the box
+        const int q = warp & 3;
+        const int m = q * 32 + lane;
+        const int per_img = p.TW * p.TH;
+        const int tn = m / per_img, rem = m - tn * per_img;
+        const int ty = rem / p.TW, txx = rem - ty * p.TW;
+        const int n = n0 + tn, y = y0 + ty, x = x0 + txx;
+        const bool pix_ok = tn < p.TN && n < p.N && y < p.H && x < p.W;
+        if (mbar_wait(bar_acc, 0, status, 3)) {
+            tc_fence_after();
+            T *out = static_cast<T *>(p.out);
+            const size_t plane = static_cast<size_t>(p.H) * p.W;
+            const size_t obase = static_cast<size_t>(n) * p.F * plane + static_cast<size_t>(y) * p.W + x;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
+                if (pix_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int f = f0 + c0 + j;
+                        if (f < p.F) {
+                            float a = __uint_as_float(v[j]) + __ldg(p.bias + f);
+                            if (p.relu) a = fmaxf(a, 0.f);
+                            if constexpr (sizeof(T) == 2) out[obase + f * plane] = __float2half_rn(a);
+                            else out[obase + f * plane] = a;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+template <int BN, int TERMS, typename T>
+cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
+    auto kern = conv_umma_kernel<BN, TERMS, T>;
+    if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+    kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
+    return cudaGetLastError();
+}
+
+cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
+#define PATDNN_UMMA(bn)                                                                          \
+    if (pl.BN == bn)                                                                             \
+        return dtype == PATDNN_F16 ? launch_umma<bn, 1, __half>(pl, p, st, prep) : launch_umma<bn, 3, float>(pl, p, st, prep);
+    PATDNN_UMMA(256) PATDNN_UMMA(128) PATDNN_UMMA(64) PATDNN_UMMA(32)
+#undef PATDNN_UMMA
+    return cudaErrorInvalidConfiguration;
+}
+
+}  // namespace
+
+bool dense_supported(int F, int C, int N, int H, int W) {
+    return encode_fn() != nullptr && F >= 1 && C >= 1 && N >= 1 && H >= 1 && W >= 1 && W <= 4096 && H <= 4096;
+}
+
+// Pixel box (TW x TH x TN <= 128) that wastes the fewest MMA rows for this image size.
+void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
+    pl = DensePlan();
+    pl.S = dtype == PATDNN_F16 ? 1 : 2;
+    pl.Cp = (C + kKBlock - 1) / kKBlock * kKBlock;
+    pl.KB = pl.Cp / kKBlock;
+    pl.BN = F > 128 ? 256 : (F > 64 ? 128 : (F > 32 ? 64 : 32));
+    pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
+    pl.n_ftiles = pl.Fp / pl.BN;
+    double best = -1;
+    for (int tw = 1; tw <= std::min(W, kTileM); ++tw) {
+        const int th = std::min(H, kTileM / tw);
+        const int tn = (th == H) ? std::max(1, std::min(N, kTileM / (tw * th))) : 1;
+        if (tw > 256 || th > 256 || tn > 256) continue;
+        const int64_t tx = (W + tw - 1) / tw, ty = (H + th - 1) / th, tz = (N + tn - 1) / tn;
+        const double util = static_cast<double>(N) * H * W / (static_cast<double>(tx * ty * tz) * kTileM);
+        const double score = util + 1e-6 * tw;                      // prefer wide boxes (coalesced stores) on ties
+        if (score > best) { best = score; pl.TW = tw; pl.TH = th; pl.TN = tn; pl.tiles_x = (int)tx; pl.tiles_y = (int)ty; pl.tiles_n = (int)tz; }
+    }
+    pl.box_bytes = pl.TW * pl.TH * pl.TN * 128;
+    const int stage = pl.S * (kTileM * 128 + pl.BN * 128);
+    pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
+    pl.smem_bytes = pl.stages * stage + 1024;
+    pl.grid = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
+}
+
+// Dense split weights [S][9][Fp][Cp] (16-bit words) from the canonical FKW arrays.
+void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16_t> &w) {
+    const size_t plane = static_cast<size_t>(9) * pl.Fp * pl.Cp;
+    w.assign(plane * pl.S, 0);
+    for (int i = 0; i < fkw.F; ++i) {
+        const int f = fkw.reorder[i];
+        for (int32_t k = fkw.offset[i]; k < fkw.offset[i + 1]; ++k) {
+            const int c = fkw.index[k];
+            const uint32_t mask = fkw.patterns[fkw.kernel_pid[k]];
+            int j = 0;
+            for (int t = 0; t < 9; ++t) {
+                if (!((mask >> t) & 1u)) continue;
+                const float v = fkw.weight_f32[static_cast<size_t>(k) * 4 + j++];
+                const size_t o = (static_cast<size_t>(t) * pl.Fp + f) * pl.Cp + c;
+                if (pl.S == 2) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+                    uint16_t hb, lb;
+                    std::memcpy(&hb, &hi, 2); std::memcpy(&lb, &lo, 2);
+                    w[o] = hb; w[plane + o] = lb;
+                } else {
+                    w[o] = float_to_half_rne(v);
+                }
+            }
+        }
+    }
+}
+
+// Tensor maps over the handle-owned split activations and weights.  Returns a PATDNN_* status.
+int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, int dtype) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return PATDNN_E_CUDA;
+    const CUtensorMapDataType dt = dtype == PATDNN_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    {
+        cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)pl.S};
+        cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)W * pl.Cp * 2, (cuuint64_t)H * W * pl.Cp * 2,
+                                 (cuuint64_t)N * H * W * pl.Cp * 2};
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)pl.TH, (cuuint32_t)pl.TN, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (enc(&pl.mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)pl.Cp, (cuuint64_t)pl.Fp, 9, (cuuint64_t)pl.S};
+        cuuint64_t strides[3] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)pl.Fp * pl.Cp * 2, (cuuint64_t)9 * pl.Fp * pl.Cp * 2};
+        cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.BN, 1, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        if (enc(&pl.mapB, dt, 4, d_w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    return PATDNN_OK;
+}
+
+cudaError_t prepare_dense(const DensePlan &pl, int dtype) {
+    DenseParams dummy{};
+    return route(pl, dummy, dtype, nullptr, true);
+}
+
+cudaError_t launch_dense(const DensePlan &pl, const DenseParams &p, const void *in, void *act, int dtype, cudaStream_t st) {
+    dim3 grid((p.W + 31) / 32, p.H, p.N), block(32, 8);
+    if (dtype == PATDNN_F16)
+        prep_act_kernel<__half><<<grid, block, 0, st>>>(static_cast<const __half *>(in), static_cast<uint16_t *>(act),
+                                                        p.N, p.C, p.H, p.W, pl.Cp, pl.S);
+    else
+        prep_act_kernel<float><<<grid, block, 0, st>>>(static_cast<const float *>(in), static_cast<uint16_t *>(act),
+                                                       p.N, p.C, p.H, p.W, pl.Cp, pl.S);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return route(pl, p, dtype, st, false);
+}
+
+}  // namespace patdnn

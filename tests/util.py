@@ -46,7 +46,7 @@ def gpu_layer(L, x=None, variant=0, order=None, via_host=False):
         xt = torch.from_numpy(x).to("cuda", dtype=tdt).contiguous()
         out = torch.full((N, L.F, H, W), float("nan"), device="cuda", dtype=tdt)
         layer.conv(xt, out, torch.cuda.current_stream().cuda_stream)
-        torch.cuda.synchronize()
+        layer.check()                 # synchronises; raises if a bounded device-side wait expired
         return out.float().cpu().numpy(), layer.plan()
     finally:
         layer.free()
