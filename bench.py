@@ -29,6 +29,9 @@ if ROOT not in sys.path:
 
 SM_COUNT, FP32_LANES, SM_MAX_GHZ = 148, 128, 1.965
 ALU_PEAK_TFLOPS = SM_COUNT * FP32_LANES * 2 * SM_MAX_GHZ / 1e3     # 74.45: FP32 FMA lanes x 2 flop x max SM clock
+# dram__bytes_read.sum + dram__bytes_write.sum of one conv_umma_kernel launch, from the ncu capture summarised under
+# profiles/ (None until a capture of the benchmark's layer shape exists)
+TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def measured_peaks():
@@ -91,6 +94,19 @@ def layer_costs(L, hbm_gbs):
     t_alu = flops / (ALU_PEAK_TFLOPS * 1e12) * 1e6
     t_hbm = byts / (hbm_gbs * 1e9) * 1e6
     return flops, byts, max(t_alu, t_hbm), ("alu" if t_alu >= t_hbm else "hbm")
+
+
+def executed_tensor_flops(L, plan):
+    """16-bit MMA flops the dense tensor-core kernel issues for a layer (0 for the CUDA-core kernels)."""
+    if plan["variant"] != 4:
+        return 0.0
+    cp = (L.C + 63) // 64 * 64
+    bn = plan["filters_per_warp"]
+    fp = (L.F + bn - 1) // bn * bn
+    ftiles = fp // bn
+    rows = plan["grid_x"] // ftiles * 128
+    terms = 1 if L.dtype == "f16" else 3
+    return terms * 2.0 * 9 * cp * fp * rows
 
 
 class VggStack:
@@ -282,6 +298,7 @@ def main():
             "layer_us": [m * 1e3 for m in layer_ms], "costs": costs, "e2e_ms": e2e_ms,
             "h2d": int(xh.numel() * 4), "d2h": int(oh.numel() * 4),
             "plans": [h.plan() for h in vs.handles], "names": [L.name for L in vs.layers],
+            "layer_objs": vs.layers,
         }
         vs.stack.free()
         for h in vs.handles:
@@ -298,6 +315,12 @@ def main():
     conv_us = sum(r["layer_us"])
     roof_us = sum(c[2] for c in r["costs"])
     achieved = r["flops"] / (conv_us * 1e-6) / 1e12
+    # dominant kernel: the tensor-core implicit GEMM (layers the planner gave to it)
+    tc = [(executed_tensor_flops(L, p), u) for L, p, u in zip(r["layer_objs"], r["plans"], r["layer_us"])]
+    tc_flops = sum(f for f, _ in tc)
+    tc_us = sum(u for f, u in tc if f > 0)
+    tc_peak = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0)))
+    tc_ach = tc_flops / (tc_us * 1e-6) / 1e12 if tc_us > 0 else 0.0
     line = {
         "metric": "effective GFLOP/s on nonzero MACs, pattern-sparse 3x3 conv", "value": world * r["flops"] / (ms * 1e-3) / 1e9,
         "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
@@ -306,20 +329,27 @@ def main():
                    "patterns": 8, "connectivity_pruning": "0% layer 1, 60% layers 2-13",
                    "l2": "working set larger than L2 (first activation alone is %d MB); input buffers rotated"
                          % (args.batch * 64 * 224 * 224 * 4 // 2**20) if args.batch >= 8 else "see batch1 leg",
-                   "step": "13 conv launches + 4 max-pool launches"},
+                   "step": "13 conv layers (tensor-core layers = layout kernel + GEMM kernel) + 4 max-pool launches"},
         "clocks": r["clocks"],
         "e2e": {"value": world * r["flops"] / (e2e_ms * 1e-3) / 1e9, "unit": "GFLOP/s",
                 "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "ms_per_step": e2e_ms},
         "gpu_launches": int(r["launches"]),
-        "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
-                     "frac": achieved / ALU_PEAK_TFLOPS, "traffic": None,
-                     "peak_source": "148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
-                     "kernel": "conv_tiled_kernel (13 launches per step, events around each launch)",
-                     "stack_roofline_us": roof_us, "stack_conv_us": conv_us, "stack_frac": roof_us / conv_us,
-                     "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
+        "roofline": {"bound": "tensor", "achieved": tc_ach, "peak": tc_peak, "unit": "TFLOP/s",
+                     "frac": tc_ach / tc_peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "peak_source": f"{peak_kind} bf16 cuBLAS peak (sustained, kernel timed inside a long step)",
+                     "kernel": "conv_umma_kernel (tcgen05 implicit GEMM, bf16 hi/lo split, 3 MMAs per product); "
+                               "achieved = executed 16-bit MMA flops / summed launch time (layout kernel included)",
+                     "launches_per_step": sum(1 for f, _ in tc if f > 0), "us_per_step": tc_us},
+        "north_star_roofline": {"definition": "per layer max(2*nonzero MACs / FP32 CUDA-core peak, algorithmic bytes / "
+                                              "measured HBM bandwidth); stack fraction = sum roofline / sum conv time",
+                                "bound": "alu", "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                                "peak_source": "148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
+                                "frac": achieved / ALU_PEAK_TFLOPS, "stack_roofline_us": roof_us,
+                                "stack_conv_us": conv_us, "stack_frac": roof_us / conv_us,
+                                "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
         "layers": [{"name": n, "us": round(u, 2), "roofline_us": round(c[2], 2), "bound": c[3],
-                    "frac": round(c[2] / u, 3), "tile": f"{p['tile_rows']}x{p['tile_cols']}x{p['filters_per_warp']}f",
-                    "grid": p["grid_x"]}
+                    "frac": round(c[2] / u, 3), "kernel": {3: "tiled", 4: "dense_tc"}.get(p["variant"], "generic"),
+                    "tile": f"{p['tile_rows']}x{p['tile_cols']}x{p['filters_per_warp']}f", "grid": p["grid_x"]}
                    for n, u, c, p in zip(r["names"], r["layer_us"], r["costs"], r["plans"])],
     }
     if rank == 0 and world == 1 and not args.no_extras:
