@@ -49,7 +49,8 @@ enum {
     PATDNN_E_DEVICE_TIMEOUT = 8,/* a bounded device-side wait expired */
     PATDNN_E_DTYPE = 9,         /* unknown dtype / variant value */
     PATDNN_E_ALLOC = 10,        /* host allocation failed */
-    PATDNN_E_STACK = 11         /* layers of a stack do not chain (shape or dtype mismatch) */
+    PATDNN_E_STACK = 11,        /* layers of a stack do not chain (shape or dtype mismatch) */
+    PATDNN_E_SCRATCH = 12       /* the layer needs more scratch than the fixed device buffer of patdnn_conv_static */
 };
 
 enum { PATDNN_F32 = 0, PATDNN_F16 = 1 };   /* storage type of weights and activations; accumulation is fp32 */
@@ -113,6 +114,28 @@ PATDNN_API int patdnn_conv(patdnn_handle h, const void *in, void *out, void *str
  * live until patdnn_free.
  */
 PATDNN_API int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void *stream);
+
+/*
+ * patdnn_conv_static -- patdnn_conv for callers that cannot allocate device memory when they run a layer: code inside
+ * a CUDA-graph replay loop or a real-time control loop, a plug-in that runs under a host whose memory pool it must
+ * not touch, or a process whose allocator is locked down after start-up.  The paper has no counterpart; this is an
+ * addition of this library.
+ *
+ * The tensor-core variant of a layer needs scratch for the re-laid-out, hi/lo-split activations.  patdnn_conv keeps
+ * that scratch in a buffer allocated by patdnn_encode; this entry point uses a fixed 16 MiB device array that is part
+ * of the library image instead, and calls no cudaMalloc, cudaFree or allocating library routine.
+ *   - in, out, stream: as for patdnn_conv (DEVICE pointers supplied by the caller).
+ *   - limit: S * N * H * W * roundup(C, 64) * 2 bytes <= 16 MiB (S = 2 for fp32 layers, 1 for fp16 layers); a larger
+ *     layer is refused with PATDNN_E_SCRATCH.  Layers that run on a CUDA-core variant need no scratch and are simply
+ *     forwarded to patdnn_conv.
+ *   - the first call on a device (and the first call for a handle) does set-up work on the host: it looks up the
+ *     device address of the array and encodes a tensor map over it.  Make that first call before starting any stream
+ *     capture.
+ *   - all calls, from every handle, share the one array, which keeps whatever the last call left in it; the kernels
+ *     overwrite everything they read, so nothing needs clearing, but two calls that can overlap on the GPU (different
+ *     streams without an ordering between them) race on the array and must be serialised by the caller.
+ */
+PATDNN_API int patdnn_conv_static(patdnn_handle h, const void *in, void *out, void *stream);
 
 /*
  * patdnn_check -- wait for the device and report whether any kernel launched for this handle gave up on a bounded

@@ -20,10 +20,10 @@ F32, F16 = 0, 1
 VARIANT_AUTO, VARIANT_NOOPT, VARIANT_REORDER, VARIANT_TILED, VARIANT_DENSE_TC = 0, 1, 2, 3, 4
 FLAG_HOST_ONLY = 1
 STATUS_NAMES = {0: "OK", 1: "E_NULL", 2: "E_SHAPE", 3: "E_PATTERN_SET", 4: "E_MASK", 5: "E_ORDER", 6: "E_CUDA",
-                7: "E_NO_DEVICE", 8: "E_DEVICE_TIMEOUT", 9: "E_DTYPE", 10: "E_ALLOC", 11: "E_STACK"}
+                7: "E_NO_DEVICE", 8: "E_DEVICE_TIMEOUT", 9: "E_DTYPE", 10: "E_ALLOC", 11: "E_STACK", 12: "E_SCRATCH"}
 
 EXPORTED_SYMBOLS = (
-    "patdnn_encode", "patdnn_conv", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
+    "patdnn_encode", "patdnn_conv", "patdnn_conv_static", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
     "patdnn_stack_free", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
     "patdnn_last_cuda_error", "patdnn_version",
@@ -75,6 +75,7 @@ def load() -> ctypes.CDLL:
                                   ctypes.POINTER(ctypes.c_uint16), i32, ctypes.POINTER(_Desc), ctypes.POINTER(vp)]
     lib.patdnn_conv.argtypes = [vp, vp, vp, vp]
     lib.patdnn_conv_host.argtypes = [vp, vp, vp, vp]
+    lib.patdnn_conv_static.argtypes = [vp, vp, vp, vp]
     lib.patdnn_free.argtypes = [vp]
     lib.patdnn_check.argtypes = [vp]
     lib.patdnn_export.argtypes = [vp, ctypes.POINTER(_FkwView)]
@@ -124,6 +125,12 @@ class Layer:
     def conv(self, x, out, stream: int = 0) -> None:
         """patdnn_conv: x, out are device buffers (NCHW); asynchronous on ``stream`` (a cudaStream_t value)."""
         _check(load().patdnn_conv(self._h, _ptr(x), _ptr(out), stream), "patdnn_conv")
+
+    def conv_static(self, x, out, stream: int = 0) -> None:
+        """patdnn_conv_static: like :meth:`conv`, but the layer's scratch is the library's fixed 16 MiB device array,
+        so the call allocates nothing (for callers that may not allocate device memory while running).  Calls that
+        can overlap on the GPU must be serialised by the caller; make the first call before any stream capture."""
+        _check(load().patdnn_conv_static(self._h, _ptr(x), _ptr(out), stream), "patdnn_conv_static")
 
     def conv_host(self, x: np.ndarray, out: np.ndarray, stream: int = 0) -> None:
         """patdnn_conv_host: host buffers in, host buffers out (copies inside the call)."""

@@ -68,6 +68,8 @@ struct patdnn_layer {
     uint16_t *d_wdense = nullptr;
     void *d_act = nullptr;
     int *d_status = nullptr;
+    DensePlan dense_static;                  // same plan with its activation map over the fixed scratch array
+    bool dense_static_ready = false;
     // staging buffers of patdnn_conv_host
     void *d_in_stage = nullptr, *d_out_stage = nullptr;
 };
@@ -250,6 +252,35 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
     }
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PATDNN_OK;
+}
+
+int patdnn_conv_static(patdnn_handle h, const void *in, void *out, void *stream) {
+    if (!h || !in || !out) return PATDNN_E_NULL;
+    if (!h->on_device) return PATDNN_E_NO_DEVICE;
+    if (h->variant != PATDNN_VARIANT_DENSE_TC) return patdnn_conv(h, in, out, stream);   // no scratch on those paths
+    const patdnn_desc &d = h->desc;
+    if (d.N == 0) return PATDNN_OK;
+    const size_t need = static_cast<size_t>(h->dense.S) * d.N * d.H * d.W * h->dense.Cp * 2;
+    if (need > kStaticScratchBytes) return PATDNN_E_SCRATCH;
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);            // first call on this device: cudaGetSymbolAddress
+    if (rc) return cuda_fail(cudaGetLastError(), "cudaGetSymbolAddress(static scratch)");
+    if (!h->dense_static_ready) {                         // first call for this handle: tensor map over the array
+        h->dense_static = h->dense;
+        rc = make_dense_maps(h->dense_static, scratch, h->d_wdense, d.N, d.H, d.W, d.dtype);
+        if (rc) return rc;
+        h->dense_static_ready = true;
+    }
+    DenseParams p{};
+    const DensePlan &pl = h->dense_static;
+    p.out = out; p.bias = h->d_bias; p.status = h->d_status;
+    p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
+    p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y;
+    p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
+    cudaError_t e = launch_dense(pl, p, in, scratch, d.dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    g_launches.fetch_add(2, std::memory_order_relaxed);
     return PATDNN_OK;
 }
 
@@ -468,6 +499,7 @@ const char *patdnn_strerror(int status) {
         case PATDNN_E_DTYPE: return "unknown dtype or variant";
         case PATDNN_E_ALLOC: return "host allocation failed";
         case PATDNN_E_STACK: return "stack layers do not chain";
+        case PATDNN_E_SCRATCH: return "layer needs more scratch than the fixed 16 MiB device buffer holds";
         default: return "unknown status";
     }
 }

@@ -111,6 +111,9 @@ struct DenseParams {
     int KB, stages, box_bytes, relu;
 };
 
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static
+int static_scratch_address(void **ptr);                    // PATDNN_* status; first call per device looks the address up
+
 bool dense_supported(int F, int C, int N, int H, int W);
 void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl);
 void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16_t> &w);

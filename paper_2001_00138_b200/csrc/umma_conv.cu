@@ -409,6 +409,28 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
     return PATDNN_OK;
 }
 
+// ---- allocation-free variant: split activations go to a fixed device array ----------------------------------------
+// Scratch for callers that must not allocate device memory at run time.  Every context that loads the library holds
+// these 16 MiB until it exits.  All calls share the array: two calls that overlap on the GPU race on it.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch for the current device.  In host code the symbol is only a handle, not an
+// address a kernel can use: the address comes from cudaGetSymbolAddress, once per device.
+int static_scratch_address(void **ptr) {
+    static void *addr[64] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= 64) return PATDNN_E_CUDA;
+    if (!addr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) return PATDNN_E_CUDA;
+        addr[dev] = p;
+    }
+    *ptr = addr[dev];
+    return PATDNN_OK;
+}
+
 cudaError_t prepare_dense(const DensePlan &pl, int dtype) {
     DenseParams dummy{};
     return route(pl, dummy, dtype, nullptr, true);
