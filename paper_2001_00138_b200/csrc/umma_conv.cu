@@ -30,6 +30,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
 
 #include "../../include/patdnn.h"
@@ -119,28 +120,52 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// ---- activation layout change + operand split ---------------------------------------------------------------------
-// grid = (ceil(W/32), H, N), block = (32, 8).  One block moves a 32-pixel row segment for all channels.
+// ---- transition into a tensor-core layer: finish the producer, change layout, split operands ---------------------
+// src is NCHW with Hs x Ws pixels: the caller's input (float or half), or the raw fp32 sums of the previous
+// tensor-core layer, in which case that layer's bias + ReLU are applied here and (clear) the sums are zeroed after
+// reading so that a K-split GEMM can accumulate into them again.  pool = 1 takes the 2x2/stride-2 maximum on the way
+// (max commutes with the per-channel bias and ReLU).  dst is [S][N][H][W][Cp], channels padded with zeros.
+// grid = (ceil(W/32), H, N * Cp/64), block = (32, 8).
 template <typename T>
-__global__ void __launch_bounds__(256) prep_act_kernel(const T *__restrict__ in, uint16_t *__restrict__ out, int N, int C,
-                                                       int H, int W, int Cp, int S) {
+__global__ void __launch_bounds__(256) transition_kernel(T *__restrict__ src, uint16_t *__restrict__ dst,
+                                                         const float *__restrict__ bias, int relu, int pool, int clear,
+                                                         int N, int C, int Hs, int Ws, int Cp, int S) {
     __shared__ float tile[64][33];
-    const int x0 = blockIdx.x * 32, y = blockIdx.y, n = blockIdx.z;
+    const int H = pool ? Hs / 2 : Hs, W = pool ? Ws / 2 : Ws;
+    const int cblocks = Cp / 64;
+    const int n = blockIdx.z / cblocks, c0 = (blockIdx.z - n * cblocks) * 64;
+    const int x0 = blockIdx.x * 32, y = blockIdx.y;
     const int tx = threadIdx.x, tyq = threadIdx.y;
     const size_t plane_out = static_cast<size_t>(N) * H * W * Cp;
-    for (int c0 = 0; c0 < Cp; c0 += 64) {
+    {
         for (int cc = tyq; cc < 64; cc += 8) {
             const int c = c0 + cc, x = x0 + tx;
             float v = 0.f;
             if (c < C && x < W) {
-                const T raw = in[((static_cast<size_t>(n) * C + c) * H + y) * W + x];
-                if constexpr (sizeof(T) == 2) v = __half2float(raw); else v = raw;
+                T *sp = src + ((static_cast<size_t>(n) * C + c) * Hs + (pool ? 2 * y : y)) * Ws + (pool ? 2 * x : x);
+                if constexpr (sizeof(T) == 2) {
+                    v = __half2float(sp[0]);
+                    if (pool) v = fmaxf(fmaxf(v, __half2float(sp[1])), fmaxf(__half2float(sp[Ws]), __half2float(sp[Ws + 1])));
+                } else {
+                    if (pool) {
+                        const float2 a = *reinterpret_cast<const float2 *>(sp), b = *reinterpret_cast<const float2 *>(sp + Ws);
+                        v = fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y));
+                        if (clear) {
+                            *reinterpret_cast<float2 *>(sp) = make_float2(0.f, 0.f);
+                            *reinterpret_cast<float2 *>(sp + Ws) = make_float2(0.f, 0.f);
+                        }
+                    } else {
+                        v = sp[0];
+                        if (clear) sp[0] = 0.f;
+                    }
+                }
+                if (bias) v += __ldg(bias + c);
+                if (relu) v = fmaxf(v, 0.f);
             }
             tile[cc][tx] = v;
         }
         __syncthreads();
-        // write: 32 pixels x 64 channels; a warp writes one pixel's 64 channels as 32 x (2 channels)
-        for (int px = tyq; px < 32; px += 8) {
+        for (int px = tyq; px < 32; px += 8) {           // a warp writes one pixel's 64 channels (2 per lane)
             const int x = x0 + px;
             if (x < W) {
                 const float a = tile[2 * tx][px], b = tile[2 * tx + 1][px];
@@ -149,20 +174,110 @@ __global__ void __launch_bounds__(256) prep_act_kernel(const T *__restrict__ in,
                     const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
                     const __nv_bfloat16 al = __float2bfloat16_rn(a - __bfloat162float(ah));
                     const __nv_bfloat16 bl = __float2bfloat16_rn(b - __bfloat162float(bh));
-                    const uint32_t hi = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) |
-                                        (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
-                    const uint32_t lo = static_cast<uint32_t>(__bfloat16_as_ushort(al)) |
-                                        (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
-                    *reinterpret_cast<uint32_t *>(out + o) = hi;
-                    *reinterpret_cast<uint32_t *>(out + plane_out + o) = lo;
+                    *reinterpret_cast<uint32_t *>(dst + o) = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) |
+                                                             (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
+                    *reinterpret_cast<uint32_t *>(dst + plane_out + o) = static_cast<uint32_t>(__bfloat16_as_ushort(al)) |
+                                                                         (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
                 } else {
-                    const uint32_t v = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(a))) |
-                                       (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(b))) << 16);
-                    *reinterpret_cast<uint32_t *>(out + o) = v;
+                    *reinterpret_cast<uint32_t *>(dst + o) = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(a))) |
+                                                             (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(b))) << 16);
                 }
             }
         }
         __syncthreads();
+    }
+}
+
+// Same operation for fp32 sources whose rows are 16-byte aligned (Ws % 4 == 0): float4 loads, 16-byte stores.
+// A block moves 64 channels x XT output pixels of one row (XT = 64, or 32 when pooling); grid = (ceil(W/XT), H, N*Cp/64).
+template <bool POOL>
+__global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__ src, uint16_t *__restrict__ dst,
+                                                             const float *__restrict__ bias, int relu, int clear,
+                                                             int N, int C, int Hs, int Ws, int Cp, int S) {
+    constexpr int XT = POOL ? 32 : 64;
+    __shared__ float tile[64][XT + 1];
+    const int H = POOL ? Hs / 2 : Hs, W = POOL ? Ws / 2 : Ws;
+    const int cblocks = Cp / 64;
+    const int n = blockIdx.z / cblocks, c0 = (blockIdx.z - n * cblocks) * 64;
+    const int x0 = blockIdx.x * XT, y = blockIdx.y;
+    const int tid = threadIdx.x;
+    const int q = tid & 15, crow = tid >> 4;                    // 16 float4 lanes per channel row, 16 rows per pass
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int cc = crow + 16 * k, c = c0 + cc;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        const int xs = (POOL ? 2 * x0 : x0) + 4 * q;             // first source column of this lane
+        if (c < C && xs < Ws) {
+            float *sp = src + ((static_cast<size_t>(n) * C + c) * Hs + (POOL ? 2 * y : y)) * Ws + xs;
+            const float4 a = *reinterpret_cast<const float4 *>(sp);
+            if (clear) *reinterpret_cast<float4 *>(sp) = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (POOL) {
+                const float4 b = *reinterpret_cast<const float4 *>(sp + Ws);
+                if (clear) *reinterpret_cast<float4 *>(sp + Ws) = make_float4(0.f, 0.f, 0.f, 0.f);
+                v[0] = fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y));
+                v[1] = fmaxf(fmaxf(a.z, a.w), fmaxf(b.z, b.w));
+            } else {
+                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+            }
+            const float bb = bias ? __ldg(bias + c) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[j] += bb;
+                if (relu) v[j] = fmaxf(v[j], 0.f);
+            }
+        }
+        if (POOL) { tile[cc][2 * q] = v[0]; tile[cc][2 * q + 1] = v[1]; }
+        else { tile[cc][4 * q] = v[0]; tile[cc][4 * q + 1] = v[1]; tile[cc][4 * q + 2] = v[2]; tile[cc][4 * q + 3] = v[3]; }
+    }
+    __syncthreads();
+    // 4 lanes per pixel, 16 channels (32 bytes) per lane per plane
+    const size_t plane_out = static_cast<size_t>(N) * H * W * Cp;
+    const int sub = tid & 3;
+#pragma unroll
+    for (int pass = 0; pass < XT / 64 + (XT < 64 ? 1 : 0); ++pass) {
+        const int px = (tid >> 2) + 64 * pass;
+        const int x = x0 + px;
+        if (px < XT && x < W) {
+            uint32_t hi[8], lo[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float a = tile[16 * sub + 2 * j][px], b = tile[16 * sub + 2 * j + 1][px];
+                if (S == 2) {
+                    const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+                    const __nv_bfloat16 al = __float2bfloat16_rn(a - __bfloat162float(ah));
+                    const __nv_bfloat16 bl = __float2bfloat16_rn(b - __bfloat162float(bh));
+                    hi[j] = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
+                    lo[j] = static_cast<uint32_t>(__bfloat16_as_ushort(al)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
+                } else {
+                    hi[j] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(a))) |
+                            (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(b))) << 16);
+                }
+            }
+            const size_t o = ((static_cast<size_t>(n) * H + y) * W + x) * Cp + c0 + 16 * sub;
+            uint4 *d0 = reinterpret_cast<uint4 *>(dst + o);
+            d0[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            d0[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+            if (S == 2) {
+                uint4 *d1 = reinterpret_cast<uint4 *>(dst + plane_out + o);
+                d1[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                d1[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+            }
+        }
+    }
+}
+
+// raw fp32 sums -> finished NCHW output of the layer (bias + ReLU), optionally zeroing the sums for the next call
+template <typename T>
+__global__ void __launch_bounds__(256) finalize_kernel(float *__restrict__ raw, T *__restrict__ out,
+                                                       const float *__restrict__ bias, int relu, int clear, int F,
+                                                       int plane, size_t total) {
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        float v = raw[i];
+        if (clear) raw[i] = 0.f;
+        v += __ldg(bias + static_cast<int>((i / plane) % F));
+        if (relu) v = fmaxf(v, 0.f);
+        if constexpr (sizeof(T) == 2) out[i] = __float2half_rn(v); else out[i] = v;
     }
 }
 
@@ -185,12 +300,16 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[8]), bar_acc = smem_u32(&bars[16]);
     int *status = p.status;
 
-    // tile coordinates: filter tile fastest so that CTAs sharing a pixel box run together (L2 reuse of the box)
+    // tile coordinates: filter tile fastest so that CTAs sharing a pixel box run together (L2 reuse of the box);
+    // the K split (a range of (channel block, tap) iterations) is slowest so that concurrent CTAs share weight tiles
     const int ft = blockIdx.x % p.n_ftiles;
     int pt = blockIdx.x / p.n_ftiles;
     const int tix = pt % p.tiles_x; pt /= p.tiles_x;
     const int tiy = pt % p.tiles_y; pt /= p.tiles_y;
-    const int x0 = tix * p.TW, y0 = tiy * p.TH, n0 = pt * p.TN, f0 = ft * BN;
+    const int tin = pt % p.tiles_n; pt /= p.tiles_n;
+    const int x0 = tix * p.TW, y0 = tiy * p.TH, n0 = tin * p.TN, f0 = ft * BN;
+    const int it0 = pt * p.iters_per_split;
+    const int iters = min(9 * p.KB, it0 + p.iters_per_split) - it0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -205,7 +324,6 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    const int iters = 9 * p.KB;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -213,7 +331,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             for (int it = 0; it < iters; ++it) {
                 const int s = it % stages, use = it / stages;
                 if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1, status, 1)) break;
-                const int cb = it / 9, tap = it - cb * 9;
+                const int cb = (it0 + it) / 9, tap = (it0 + it) - cb * 9;
                 const int r = tap / 3, sx = tap - 3 * r;
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
                 mbar_expect_tx(bar_full + 8 * s, tx_bytes);
@@ -260,7 +378,6 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const bool pix_ok = tn < p.TN && n < p.N && y < p.H && x < p.W;
         if (mbar_wait(bar_acc, 0, status, 3)) {
             tc_fence_after();
-            T *out = static_cast<T *>(p.out);
             const size_t plane = static_cast<size_t>(p.H) * p.W;
             const size_t obase = static_cast<size_t>(n) * p.F * plane + static_cast<size_t>(y) * p.W + x;
 #pragma unroll 1
@@ -268,14 +385,27 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 uint32_t v[32];
                 tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
                 if (pix_ok) {
+                    if (p.mode == 0) {                      // finished layer: bias + ReLU, caller's NCHW tensor
+                        T *out = static_cast<T *>(p.out);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int f = f0 + c0 + j;
-                        if (f < p.F) {
-                            float a = __uint_as_float(v[j]) + __ldg(p.bias + f);
-                            if (p.relu) a = fmaxf(a, 0.f);
-                            if constexpr (sizeof(T) == 2) out[obase + f * plane] = __float2half_rn(a);
-                            else out[obase + f * plane] = a;
+                        for (int j = 0; j < 32; ++j) {
+                            const int f = f0 + c0 + j;
+                            if (f < p.F) {
+                                float a = __uint_as_float(v[j]) + __ldg(p.bias + f);
+                                if (p.relu) a = fmaxf(a, 0.f);
+                                if constexpr (sizeof(T) == 2) out[obase + f * plane] = __float2half_rn(a);
+                                else out[obase + f * plane] = a;
+                            }
+                        }
+                    } else {                                // raw sums (fp32 NCHW): plain store, or add when K is split
+                        float *raw = p.raw;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int f = f0 + c0 + j;
+                            if (f < p.F) {
+                                if (p.mode == 1) raw[obase + f * plane] = __uint_as_float(v[j]);
+                                else atomicAdd(raw + obase + f * plane, __uint_as_float(v[j]));
+                            }
                         }
                     }
                 }
@@ -347,11 +477,21 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
         const double score = util + 1e-6 * tw;                      // prefer wide boxes (coalesced stores) on ties
         if (score > best) { best = score; pl.TW = tw; pl.TH = th; pl.TN = tn; pl.tiles_x = (int)tx; pl.tiles_y = (int)ty; pl.tiles_n = (int)tz; }
     }
+    // Few pixel tiles (small batch): keep the filter tile wide (every A byte then feeds more MMA work) and cut the
+    // K loop into ranges until the grid fills the GPU; the ranges are summed with atomic adds.
+    const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
+    const int total_iters = 9 * pl.KB;
+    int ks = 1;
+    const int base_grid = ptiles * pl.n_ftiles;
+    if (base_grid < 100) ks = std::max(1, std::min(total_iters / 2, (280 + base_grid / 2) / base_grid));   // ~2 waves
+    if (const char *ov = std::getenv("PATDNN_KSPLIT")) ks = std::max(1, std::min(total_iters, atoi(ov)));
+    pl.iters_per_split = (total_iters + ks - 1) / ks;
+    pl.ksplit = (total_iters + pl.iters_per_split - 1) / pl.iters_per_split;
     pl.box_bytes = pl.TW * pl.TH * pl.TN * 128;
     const int stage = pl.S * (kTileM * 128 + pl.BN * 128);
     pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
     pl.smem_bytes = pl.stages * stage + 1024;
-    pl.grid = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
+    pl.grid = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles * pl.ksplit;
 }
 
 // Dense split weights [S][9][Fp][Cp] (16-bit words) from the canonical FKW arrays.
@@ -436,16 +576,44 @@ cudaError_t prepare_dense(const DensePlan &pl, int dtype) {
     return route(pl, dummy, dtype, nullptr, true);
 }
 
-cudaError_t launch_dense(const DensePlan &pl, const DenseParams &p, const void *in, void *act, int dtype, cudaStream_t st) {
-    dim3 grid((p.W + 31) / 32, p.H, p.N), block(32, 8);
-    if (dtype == PATDNN_F16)
-        prep_act_kernel<__half><<<grid, block, 0, st>>>(static_cast<const __half *>(in), static_cast<uint16_t *>(act),
-                                                        p.N, p.C, p.H, p.W, pl.Cp, pl.S);
+cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const float *bias, int relu, int pool, int clear,
+                              int N, int C, int Hs, int Ws, int Cp, int S, cudaStream_t st) {
+    const int H = pool ? Hs / 2 : Hs, W = pool ? Ws / 2 : Ws;
+    if (N == 0 || H == 0 || W == 0) return cudaSuccess;
+    const int gz = N * (Cp / 64);
+    if (!src_is_half && Ws % 4 == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+        float *fs = static_cast<float *>(const_cast<void *>(src));
+        if (pool)
+            transition_vec_kernel<true><<<dim3((W + 31) / 32, H, gz), 256, 0, st>>>(fs, static_cast<uint16_t *>(dst), bias, relu,
+                                                                                     clear, N, C, Hs, Ws, Cp, S);
+        else
+            transition_vec_kernel<false><<<dim3((W + 63) / 64, H, gz), 256, 0, st>>>(fs, static_cast<uint16_t *>(dst), bias, relu,
+                                                                                      clear, N, C, Hs, Ws, Cp, S);
+        return cudaGetLastError();
+    }
+    dim3 grid((W + 31) / 32, H, gz), block(32, 8);
+    if (src_is_half)
+        transition_kernel<__half><<<grid, block, 0, st>>>(static_cast<__half *>(const_cast<void *>(src)),
+                                                          static_cast<uint16_t *>(dst), bias, relu, pool, 0, N, C, Hs, Ws, Cp, S);
     else
-        prep_act_kernel<float><<<grid, block, 0, st>>>(static_cast<const float *>(in), static_cast<uint16_t *>(act),
-                                                       p.N, p.C, p.H, p.W, pl.Cp, pl.S);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+        transition_kernel<float><<<grid, block, 0, st>>>(static_cast<float *>(const_cast<void *>(src)),
+                                                         static_cast<uint16_t *>(dst), bias, relu, pool, clear, N, C, Hs, Ws, Cp, S);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(float *raw, void *out, int dtype, const float *bias, int relu, int clear, int N, int F, int H,
+                            int W, cudaStream_t st) {
+    const size_t total = static_cast<size_t>(N) * F * H * W;
+    if (total == 0) return cudaSuccess;
+    const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 16));
+    if (dtype == PATDNN_F16)
+        finalize_kernel<__half><<<blocks, 256, 0, st>>>(raw, static_cast<__half *>(out), bias, relu, clear, F, H * W, total);
+    else
+        finalize_kernel<float><<<blocks, 256, 0, st>>>(raw, static_cast<float *>(out), bias, relu, clear, F, H * W, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dense_gemm(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st) {
     return route(pl, p, dtype, st, false);
 }
 

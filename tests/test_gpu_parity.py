@@ -147,7 +147,7 @@ def test_vgg_stack_reduced_spatial_per_layer_and_chained():
     assert_close(out.cpu().numpy(), cur, 10 * TOL_F32, "vgg chained")      # 13 layers of rounding compound
     out_h = np.empty(cur.shape, dtype=np.float32)
     stack.run_host(x, out_h)
-    assert np.array_equal(out_h, out.cpu().numpy())
+    assert_close(out_h, cur, 10 * TOL_F32, "vgg chained through host buffers")   # K-split sums are order-free
     stack.free()
     for h in handles:
         h.free()
