@@ -104,7 +104,7 @@ def executed_tensor_flops(L, plan):
     bn = plan["filters_per_warp"]
     fp = (L.F + bn - 1) // bn * bn
     ftiles = fp // bn
-    rows = plan["grid_x"] // ftiles * 128
+    rows = plan["grid_x"] // (ftiles * max(plan["channel_splits"], 1)) * 128
     terms = 1 if L.dtype == "f16" else 3
     return terms * 2.0 * 9 * cp * fp * rows
 

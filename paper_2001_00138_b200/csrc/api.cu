@@ -68,7 +68,6 @@ struct patdnn_layer {
     uint16_t *d_wdense = nullptr;
     void *d_act = nullptr;
     int *d_status = nullptr;
-    float *d_raw = nullptr;                  // fp32 NCHW sums of a K-split GEMM / of a layer inside a stack
     DensePlan dense_static;                  // same plan with its activation map over the fixed scratch array
     bool dense_static_ready = false;
     // staging buffers of patdnn_conv_host
@@ -86,18 +85,6 @@ struct patdnn_stack_s {
 
 static size_t esize_of(int dtype) { return dtype == PATDNN_F16 ? 2 : 4; }
 
-static int ensure_raw(patdnn_layer *h) {
-    if (h->d_raw) return PATDNN_OK;
-    const patdnn_desc &d = h->desc;
-    const size_t bytes = std::max<size_t>(static_cast<size_t>(std::max(d.N, 1)) * d.F * d.H * d.W * 4, 16);
-    void *p = nullptr;
-    CU(cudaMalloc(&p, bytes));
-    h->owned.push_back(p);
-    CU(cudaMemset(p, 0, bytes));
-    h->d_raw = static_cast<float *>(p);
-    return PATDNN_OK;
-}
-
 static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
     const patdnn_desc &d = h->desc;
     DenseParams p{};
@@ -105,20 +92,19 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
     p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
     p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y; p.tiles_n = pl.tiles_n;
     p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
-    p.iters_per_split = pl.iters_per_split;
+    p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit;
     return p;
 }
 
 // GEMM of a tensor-core layer whose split activations already sit in the buffer its activation map points to.
-// to_raw: leave the raw sums in h->d_raw (a stack transition or a finalize pass finishes the layer).
-static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, bool to_raw, cudaStream_t st) {
+// next == nullptr: finished NCHW result into `out`; else the result goes, already split and channels-innermost, straight
+// into the activation buffer of the tensor-core layer `next` (same spatial size, no pooling in between).
+static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const patdnn_layer *next, cudaStream_t st) {
     DenseParams p = dense_params(h, pl);
-    if (to_raw || pl.ksplit > 1) {
-        p.mode = pl.ksplit > 1 ? 2 : 1;
-        p.raw = h->d_raw;
+    if (next) {
+        p.mode = 3; p.out = next->d_act; p.out_cp = next->dense.Cp;
     } else {
-        p.mode = 0;
-        p.out = out;
+        p.mode = 0; p.out = out;
     }
     cudaError_t e = launch_dense_gemm(pl, p, h->desc.dtype, st);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core kernel launch");
@@ -132,14 +118,7 @@ static int dense_forward(patdnn_layer *h, const DensePlan &pl, const void *in, v
     cudaError_t e = launch_transition(in, d.dtype == PATDNN_F16, act, nullptr, 0, 0, 0, d.N, d.C, d.H, d.W, pl.Cp, pl.S, st);
     if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    int rc = dense_gemm(h, pl, out, false, st);
-    if (rc) return rc;
-    if (pl.ksplit > 1) {
-        e = launch_finalize(h->d_raw, out, d.dtype, h->d_bias, d.relu, 1, d.N, d.F, d.H, d.W, st);
-        if (e != cudaSuccess) return cuda_fail(e, "finalize kernel launch");
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-    }
-    return PATDNN_OK;
+    return dense_gemm(h, pl, out, nullptr, st);
 }
 
 extern "C" {
@@ -215,13 +194,17 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                                                  desc->W * h->dense.Cp * 2;
                         cudaError_t ce = cudaMalloc(&h->d_act, act_bytes);
                         if (ce != cudaSuccess) rc = cuda_fail(ce, "cudaMalloc(split activations)");
-                        else h->owned.push_back(h->d_act);
+                        else {
+                            h->owned.push_back(h->d_act);
+                            // padded channels must read as zero even when a producer writes fewer channels than Cp
+                            ce = cudaMemset(h->d_act, 0, act_bytes);
+                            if (ce != cudaSuccess) rc = cuda_fail(ce, "cudaMemset(split activations)");
+                        }
                     }
                     if (!rc) {
                         std::vector<int> zero(4, 0);
                         rc = upload(zero, &h->d_status, h->owned);
                     }
-                    if (!rc && h->dense.ksplit > 1) rc = ensure_raw(h);
                     if (!rc) rc = make_dense_maps(h->dense, h->d_act, h->d_wdense, std::max(desc->N, 1), desc->H, desc->W, desc->dtype);
                     if (rc == PATDNN_E_CUDA && g_cuda_error.empty()) g_cuda_error = "cuTensorMapEncodeTiled failed";
                     if (!rc) {
@@ -408,7 +391,7 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
     } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         const DensePlan &p = h->dense;
         info->tile_rows = p.TH; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
-        info->channels_per_stage = 64; info->channel_splits = 1;
+        info->channels_per_stage = 64; info->channel_splits = p.ksplit;
         info->grid_x = p.grid; info->grid_y = 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
         info->entries = static_cast<int64_t>(9) * p.Fp * p.Cp;
     } else {
@@ -454,10 +437,6 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         }
         s->layers.push_back(h);
         s->pool.push_back(pool);
-        if (h->variant == PATDNN_VARIANT_DENSE_TC) {       // inside a stack a tensor-core layer leaves raw sums behind
-            const int rc = ensure_raw(h);
-            if (rc) { delete s; return rc; }
-        }
     }
     s->oN = N; s->oF = C; s->oH = H; s->oW = W;
     s->buf_bytes = std::max<size_t>(max_bytes, 16);
@@ -472,83 +451,58 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
     return PATDNN_OK;
 }
 
-// Chained execution.  Between two tensor-core layers nothing is written in finished NCHW form: the first leaves its raw
-// fp32 sums, and ONE transition kernel applies its bias + ReLU, the optional 2x2 max-pool, the layout change and the
-// operand split for the second.  CUDA-core layers (and the stack's ends) use finished NCHW tensors.
+// Chained execution.  Where two tensor-core layers follow each other without a pool, the first one's epilogue writes
+// the second one's input directly (bias + ReLU applied, channels innermost, operands split): no tensor in NCHW form and
+// no layout kernel in between.  A pool between them is folded into the layout kernel of the second.
 int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
     if (!s || !in || !out) return PATDNN_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n = static_cast<int>(s->layers.size());
-    const void *cur = in;            // finished NCHW activations (valid when pending == nullptr)
+    const void *cur = in;            // finished NCHW activations feeding the next layer (unless `direct`)
     bool cur_pool = false;           // a 2x2 max-pool still has to be applied to `cur`
-    patdnn_layer *pending = nullptr; // tensor-core layer whose raw sums wait to be finished
-    bool pending_pool = false;
+    bool direct = false;             // the next layer's split input was already written by the previous epilogue
     int which = 0;
-    auto finish_pending = [&](void *dst) -> int {        // raw sums -> finished NCHW in dst (pool not applied)
-        const patdnn_desc &d = pending->desc;
-        cudaError_t e = launch_finalize(pending->d_raw, dst, d.dtype, pending->d_bias, d.relu, pending->dense.ksplit > 1,
-                                        d.N, d.F, d.H, d.W, st);
-        if (e != cudaSuccess) return cuda_fail(e, "finalize kernel launch");
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        return PATDNN_OK;
-    };
+    int curH = s->layers[0]->desc.H, curW = s->layers[0]->desc.W;   // spatial size of `cur` (before a pending pool)
     for (int i = 0; i < n; ++i) {
         patdnn_layer *h = s->layers[i];
         const patdnn_desc &d = h->desc;
         if (d.N == 0) return PATDNN_OK;
-        if (h->variant == PATDNN_VARIANT_DENSE_TC) {
-            cudaError_t e;
-            if (pending) {
-                const patdnn_desc &pd = pending->desc;
-                e = launch_transition(pending->d_raw, 0, h->d_act, pending->d_bias, pd.relu, pending_pool,
-                                      pending->dense.ksplit > 1, pd.N, pd.F, pd.H, pd.W, h->dense.Cp, h->dense.S, st);
-            } else {
-                e = launch_transition(cur, d.dtype == PATDNN_F16, h->d_act, nullptr, 0, cur_pool, 0, d.N, d.C,
-                                      cur_pool ? d.H * 2 : d.H, cur_pool ? d.W * 2 : d.W, h->dense.Cp, h->dense.S, st);
+        const bool last = (i == n - 1);
+        const bool is_dense = h->variant == PATDNN_VARIANT_DENSE_TC;
+        if (is_dense) {
+            if (!direct) {
+                cudaError_t e = launch_transition(cur, d.dtype == PATDNN_F16, h->d_act, nullptr, 0, cur_pool, 0, d.N, d.C,
+                                                  curH, curW, h->dense.Cp, h->dense.S, st);
+                if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
+                g_launches.fetch_add(1, std::memory_order_relaxed);
             }
-            if (e != cudaSuccess) return cuda_fail(e, "transition kernel launch");
-            g_launches.fetch_add(1, std::memory_order_relaxed);
-            const int rc = dense_gemm(h, h->dense, nullptr, true, st);
+            patdnn_layer *next = (!last && !s->pool[i] && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC)
+                                     ? s->layers[i + 1] : nullptr;
+            void *dst = next ? nullptr : ((last && !s->pool[i]) ? out : s->buf[which]);
+            const int rc = dense_gemm(h, h->dense, dst, next, st);
             if (rc) return rc;
-            pending = h;
-            pending_pool = s->pool[i] != 0;
-            cur_pool = false;
+            direct = next != nullptr;
+            if (!direct) { cur = dst; which ^= 1; }
+            cur_pool = s->pool[i] != 0;
+            curH = d.H; curW = d.W;
         } else {
-            if (pending) {                                 // finish the tensor-core layer into a stack buffer
-                const patdnn_desc &pd = pending->desc;
-                int rc = finish_pending(s->buf[which]);
+            if (cur_pool) {
+                const int rc = patdnn_maxpool2x2(cur, s->buf[which], d.N, d.C, curH, curW, d.dtype, stream);
                 if (rc) return rc;
                 cur = s->buf[which];
                 which ^= 1;
-                if (pending_pool) {
-                    rc = patdnn_maxpool2x2(cur, s->buf[which], pd.N, pd.F, pd.H, pd.W, pd.dtype, stream);
-                    if (rc) return rc;
-                    cur = s->buf[which];
-                    which ^= 1;
-                }
-                pending = nullptr;
-            } else if (cur_pool) {
-                const int rc = patdnn_maxpool2x2(cur, s->buf[which], d.N, d.C, d.H * 2, d.W * 2, d.dtype, stream);
-                if (rc) return rc;
-                cur = s->buf[which];
-                which ^= 1;
-                cur_pool = false;
             }
-            const bool last = (i == n - 1);
             void *dst = (last && !s->pool[i]) ? out : s->buf[which];
             const int rc = patdnn_conv(h, cur, dst, stream);
             if (rc) return rc;
             cur = dst;
             which ^= 1;
             cur_pool = s->pool[i] != 0;
+            curH = d.H; curW = d.W;
+            direct = false;
         }
     }
-    if (pending) {
-        const patdnn_desc &pd = pending->desc;
-        int rc = finish_pending(pending_pool ? s->buf[which] : out);
-        if (rc) return rc;
-        if (pending_pool) return patdnn_maxpool2x2(s->buf[which], out, pd.N, pd.F, pd.H, pd.W, pd.dtype, stream);
-    } else if (cur_pool) {
+    if (cur_pool) {
         const patdnn_desc &ld = s->layers[n - 1]->desc;
         return patdnn_maxpool2x2(cur, out, ld.N, ld.F, ld.H, ld.W, ld.dtype, stream);
     }

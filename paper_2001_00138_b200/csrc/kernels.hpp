@@ -99,7 +99,7 @@ struct DensePlan {
     int TW = 0, TH = 0, TN = 0; // pixel box (columns, rows, images), TW*TH*TN <= 128
     int tiles_x = 0, tiles_y = 0, tiles_n = 0;
     int box_bytes = 0, stages = 0, smem_bytes = 0, grid = 0;
-    int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges, summed with atomics
+    int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
     CUtensorMap mapA{}, mapB{};
 };
 
@@ -110,9 +110,9 @@ struct DenseParams {
     int N, C, H, W, F;
     int TW, TH, TN, tiles_x, tiles_y, n_ftiles;
     int KB, stages, box_bytes, relu;
-    int tiles_n, iters_per_split;
-    int mode;                   // 0: bias + ReLU -> out (NCHW); 1: raw sums -> raw (store); 2: raw sums -> raw (atomic add)
-    float *raw;                 // fp32 NCHW sums (modes 1, 2)
+    int tiles_n, iters_per_split, ksplit;
+    int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer
+    int out_cp;                 // channel pitch of the mode-3 destination
 };
 
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static
@@ -125,8 +125,6 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
 cudaError_t prepare_dense(const DensePlan &pl, int dtype);
 cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const float *bias, int relu, int pool, int clear,
                               int N, int C, int Hs, int Ws, int Cp, int S, cudaStream_t st);
-cudaError_t launch_finalize(float *raw, void *out, int dtype, const float *bias, int relu, int clear, int N, int F, int H,
-                            int W, cudaStream_t st);
 cudaError_t launch_dense_gemm(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st);
 
 }  // namespace patdnn

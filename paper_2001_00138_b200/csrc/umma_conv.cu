@@ -266,18 +266,56 @@ __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__
     }
 }
 
-// raw fp32 sums -> finished NCHW output of the layer (bias + ReLU), optionally zeroing the sums for the next call
-template <typename T>
-__global__ void __launch_bounds__(256) finalize_kernel(float *__restrict__ raw, T *__restrict__ out,
-                                                       const float *__restrict__ bias, int relu, int clear, int F,
-                                                       int plane, size_t total) {
-    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        float v = raw[i];
-        if (clear) raw[i] = 0.f;
-        v += __ldg(bias + static_cast<int>((i / plane) % F));
-        if (relu) v = fmaxf(v, 0.f);
-        if constexpr (sizeof(T) == 2) out[i] = __float2half_rn(v); else out[i] = v;
+// Finish CNT consecutive filters (f_lo ..) of one output pixel: bias + ReLU, then either the caller's NCHW tensor
+// (mode 0) or the next tensor-core layer's split channels-innermost activations (mode 3: [S][N][H][W][out_cp]).
+template <int CNT, typename T>
+__device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT], int f_lo, int n, int y, int x, bool pix_ok) {
+#pragma unroll
+    for (int j = 0; j < CNT; ++j) {
+        const int f = f_lo + j;
+        float v = (f < p.F) ? a[j] + __ldg(p.bias + f) : 0.f;
+        if (p.relu) v = fmaxf(v, 0.f);
+        a[j] = (f < p.F) ? v : 0.f;
+    }
+    if (!pix_ok) return;
+    if (p.mode == 0) {
+        T *out = static_cast<T *>(p.out);
+        const size_t plane = static_cast<size_t>(p.H) * p.W;
+        const size_t obase = static_cast<size_t>(n) * p.F * plane + static_cast<size_t>(y) * p.W + x;
+#pragma unroll
+        for (int j = 0; j < CNT; ++j) {
+            const int f = f_lo + j;
+            if (f < p.F) {
+                if constexpr (sizeof(T) == 2) out[obase + f * plane] = __float2half_rn(a[j]);
+                else out[obase + f * plane] = a[j];
+            }
+        }
+    } else {
+        if (f_lo >= p.out_cp) return;                    // filter tiles may be padded beyond the next layer's channels
+        uint16_t *dst = static_cast<uint16_t *>(p.out);
+        const size_t o = ((static_cast<size_t>(n) * p.H + y) * p.W + x) * p.out_cp + f_lo;
+        const size_t plane_out = static_cast<size_t>(p.N) * p.H * p.W * p.out_cp;
+#pragma unroll
+        for (int g = 0; g < CNT / 8; ++g) {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float u = a[8 * g + 2 * j], w = a[8 * g + 2 * j + 1];
+                if constexpr (sizeof(T) == 2) {
+                    hi[j] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(u))) |
+                            (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(w))) << 16);
+                    lo[j] = 0;
+                } else {
+                    const __nv_bfloat16 uh = __float2bfloat16_rn(u), wh = __float2bfloat16_rn(w);
+                    const __nv_bfloat16 ul = __float2bfloat16_rn(u - __bfloat162float(uh));
+                    const __nv_bfloat16 wl = __float2bfloat16_rn(w - __bfloat162float(wh));
+                    hi[j] = static_cast<uint32_t>(__bfloat16_as_ushort(uh)) | (static_cast<uint32_t>(__bfloat16_as_ushort(wh)) << 16);
+                    lo[j] = static_cast<uint32_t>(__bfloat16_as_ushort(ul)) | (static_cast<uint32_t>(__bfloat16_as_ushort(wl)) << 16);
+                }
+            }
+            *reinterpret_cast<uint4 *>(dst + o + 8 * g) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            if constexpr (sizeof(T) != 2) *reinterpret_cast<uint4 *>(dst + plane_out + o + 8 * g) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
     }
 }
 
@@ -300,16 +338,26 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[8]), bar_acc = smem_u32(&bars[16]);
     int *status = p.status;
 
-    // tile coordinates: filter tile fastest so that CTAs sharing a pixel box run together (L2 reuse of the box);
-    // the K split (a range of (channel block, tap) iterations) is slowest so that concurrent CTAs share weight tiles
-    const int ft = blockIdx.x % p.n_ftiles;
-    int pt = blockIdx.x / p.n_ftiles;
+    // The ks CTAs of a cluster share one (pixel box, filter tile) and split its K loop -- the (channel block, tap)
+    // iterations -- into ks ranges; then the filter tile index is fastest so that CTAs sharing a pixel box run together.
+    const int ks = p.ksplit;
+    const int rank = blockIdx.x % ks;
+    int pt = blockIdx.x / ks;
+    const int ft = pt % p.n_ftiles; pt /= p.n_ftiles;
     const int tix = pt % p.tiles_x; pt /= p.tiles_x;
     const int tiy = pt % p.tiles_y; pt /= p.tiles_y;
-    const int tin = pt % p.tiles_n; pt /= p.tiles_n;
+    const int tin = pt;
     const int x0 = tix * p.TW, y0 = tiy * p.TH, n0 = tin * p.TN, f0 = ft * BN;
-    const int it0 = pt * p.iters_per_split;
-    const int iters = min(9 * p.KB, it0 + p.iters_per_split) - it0;
+    const int it0 = rank * (9 * p.KB) / ks;                     // even split: every range holds at least one iteration
+    const int iters = (rank + 1) * (9 * p.KB) / ks - it0;
+    // output pixel of this thread when it acts as an epilogue thread (warps 2..5 cover the 128 accumulator rows)
+    const int q = warp & 3;
+    const int m = q * 32 + lane;
+    const int per_img = p.TW * p.TH;
+    const int tn = m / per_img, rem = m - tn * per_img;
+    const int ty = rem / p.TW, txx = rem - ty * p.TW;
+    const int n = n0 + tn, y = y0 + ty, x = x0 + txx;
+    const bool pix_ok = tn < p.TN && n < p.N && y < p.H && x < p.W;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -368,49 +416,59 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (ok) umma_commit(bar_acc);
         }
     } else {
-        // epilogue: warp w reads TMEM lanes 32*(w%4) .. +31; lane = output pixel of the box
-        const int q = warp & 3;
-        const int m = q * 32 + lane;
-        const int per_img = p.TW * p.TH;
-        const int tn = m / per_img, rem = m - tn * per_img;
-        const int ty = rem / p.TW, txx = rem - ty * p.TW;
-        const int n = n0 + tn, y = y0 + ty, x = x0 + txx;
-        const bool pix_ok = tn < p.TN && n < p.N && y < p.H && x < p.W;
+        // epilogue warps: warp w owns TMEM lanes 32*(w%4) .. +31; lane = output pixel m of the box
         if (mbar_wait(bar_acc, 0, status, 3)) {
             tc_fence_after();
-            const size_t plane = static_cast<size_t>(p.H) * p.W;
-            const size_t obase = static_cast<size_t>(n) * p.F * plane + static_cast<size_t>(y) * p.W + x;
+            if (ks == 1) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
-                if (pix_ok) {
-                    if (p.mode == 0) {                      // finished layer: bias + ReLU, caller's NCHW tensor
-                        T *out = static_cast<T *>(p.out);
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
+                    float a[32];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int f = f0 + c0 + j;
-                            if (f < p.F) {
-                                float a = __uint_as_float(v[j]) + __ldg(p.bias + f);
-                                if (p.relu) a = fmaxf(a, 0.f);
-                                if constexpr (sizeof(T) == 2) out[obase + f * plane] = __float2half_rn(a);
-                                else out[obase + f * plane] = a;
-                            }
-                        }
-                    } else {                                // raw sums (fp32 NCHW): plain store, or add when K is split
-                        float *raw = p.raw;
+                    for (int j = 0; j < 32; ++j) a[j] = __uint_as_float(v[j]);
+                    emit_chunk<32, T>(p, a, f0 + c0, n, y, x, pix_ok);
+                }
+            } else {
+                // partial sums of this K range -> own shared memory, column-major [BN][128] (pipeline buffers are free)
+                float *R = reinterpret_cast<float *>(smem);
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int f = f0 + c0 + j;
-                            if (f < p.F) {
-                                if (p.mode == 1) raw[obase + f * plane] = __uint_as_float(v[j]);
-                                else atomicAdd(raw + obase + f * plane, __uint_as_float(v[j]));
-                            }
-                        }
-                    }
+                    for (int j = 0; j < 32; ++j) R[(c0 + j) * kTileM + m] = __uint_as_float(v[j]);
                 }
             }
         }
+    }
+    if (ks > 1) {
+        // Sum the K ranges across the cluster through distributed shared memory: CTA r finishes columns
+        // [r*BN/ks, (r+1)*BN/ks).  Every thread of every CTA takes part in both cluster barriers, also after a
+        // timed-out wait, so nobody is left waiting.
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (warp >= 2) {
+            const int cols = BN / ks, cbeg = rank * cols;
+            const uint32_t rbase = smem_u32(smem);
+#pragma unroll 1
+            for (int c0 = 0; c0 < cols; c0 += 8) {
+                float a[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) a[j] = 0.f;
+                for (int qq = 0; qq < ks; ++qq) {
+                    uint32_t remote;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(rbase), "r"(qq));
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float t;
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(t) : "r"(remote + ((cbeg + c0 + j) * kTileM + m) * 4) : "memory");
+                        a[j] += t;
+                    }
+                }
+                emit_chunk<8, T>(p, a, f0 + cbeg + c0, n, y, x, pix_ok);
+            }
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
@@ -439,8 +497,17 @@ template <int BN, int TERMS, typename T>
 cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_kernel<BN, TERMS, T>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
-    kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
-    return cudaGetLastError();
+    if (pl.ksplit == 1) {
+        kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = pl.smem_bytes; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pl.ksplit; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, pl.mapA, pl.mapB, p);
 }
 
 cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
@@ -477,16 +544,24 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
         const double score = util + 1e-6 * tw;                      // prefer wide boxes (coalesced stores) on ties
         if (score > best) { best = score; pl.TW = tw; pl.TH = th; pl.TN = tn; pl.tiles_x = (int)tx; pl.tiles_y = (int)ty; pl.tiles_n = (int)tz; }
     }
-    // Few pixel tiles (small batch): keep the filter tile wide (every A byte then feeds more MMA work) and cut the
-    // K loop into ranges until the grid fills the GPU; the ranges are summed with atomic adds.
+    // Few pixel tiles (small batch): cut the K loop into ks ranges, one CTA each, ks CTAs forming a cluster that sums
+    // its partial tiles through distributed shared memory; only when even 8 ranges leave most SMs idle, narrow the
+    // filter tile as well (a wide tile makes every loaded activation byte feed more MMA work).
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
     const int total_iters = 9 * pl.KB;
-    int ks = 1;
+    while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 8 < 120) pl.BN /= 2;
+    pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
+    pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
-    if (base_grid < 100) ks = std::max(1, std::min(total_iters / 2, (280 + base_grid / 2) / base_grid));   // ~2 waves
-    if (const char *ov = std::getenv("PATDNN_KSPLIT")) ks = std::max(1, std::min(total_iters, atoi(ov)));
+    int ks = 1;
+    if (base_grid < 100)
+        while (ks < 8 && base_grid * ks * 2 <= 296 && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
+    if (const char *ov = std::getenv("PATDNN_KSPLIT")) {
+        const int want = atoi(ov);
+        if ((want == 1 || want == 2 || want == 4 || want == 8) && want <= total_iters && pl.BN / want >= 8) ks = want;
+    }
+    pl.ksplit = ks;
     pl.iters_per_split = (total_iters + ks - 1) / ks;
-    pl.ksplit = (total_iters + pl.iters_per_split - 1) / pl.iters_per_split;
     pl.box_bytes = pl.TW * pl.TH * pl.TN * 128;
     const int stage = pl.S * (kTileM * 128 + pl.BN * 128);
     pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
@@ -598,18 +673,6 @@ cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const
     else
         transition_kernel<float><<<grid, block, 0, st>>>(static_cast<float *>(const_cast<void *>(src)),
                                                          static_cast<uint16_t *>(dst), bias, relu, pool, clear, N, C, Hs, Ws, Cp, S);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_finalize(float *raw, void *out, int dtype, const float *bias, int relu, int clear, int N, int F, int H,
-                            int W, cudaStream_t st) {
-    const size_t total = static_cast<size_t>(N) * F * H * W;
-    if (total == 0) return cudaSuccess;
-    const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 16));
-    if (dtype == PATDNN_F16)
-        finalize_kernel<__half><<<blocks, 256, 0, st>>>(raw, static_cast<__half *>(out), bias, relu, clear, F, H * W, total);
-    else
-        finalize_kernel<float><<<blocks, 256, 0, st>>>(raw, static_cast<float *>(out), bias, relu, clear, F, H * W, total);
     return cudaGetLastError();
 }
 

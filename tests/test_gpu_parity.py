@@ -179,6 +179,20 @@ def test_vgg_full_size_sampled(i, N):
     layer.free()
 
 
+@pytest.mark.parametrize("ks", [1, 2, 4, 8])
+def test_tensor_core_path_with_cluster_split_of_the_channel_loop(ks, monkeypatch):
+    """Small batches split the (channel block, tap) loop over the CTAs of a cluster and sum through distributed shared
+    memory; every split factor must give the same layer."""
+    monkeypatch.setenv("PATDNN_KSPLIT", str(ks))
+    L = synth.make_layer("ks", F=192, C=160, N=1, H=20, W=24, seed=900 + ks, prune=0.6, bias_std=0.1, x_dist="normal")
+    got, plan = gpu_layer(L, variant=VARIANTS["dense"])
+    assert plan["variant"] == 4
+    assert_close(got, oracle_layer(L), TOL_F32, f"cluster split {ks}")
+    Lh = synth.resnet50_layer(1, N=2)
+    got, _ = gpu_layer(Lh, variant=VARIANTS["dense"])
+    assert_close(got, oracle_layer(Lh), TOL_F16, f"cluster split {ks}, fp16")
+
+
 def test_maxpool_matches_oracle():
     import oracle
     import torch
