@@ -104,7 +104,8 @@ def executed_tensor_flops(L, plan):
     bn = plan["filters_per_warp"]
     fp = (L.F + bn - 1) // bn * bn
     ftiles = fp // bn
-    rows = plan["grid_x"] // (ftiles * max(plan["channel_splits"], 1)) * 128
+    ctas = plan["grid_y"] if plan["grid_y"] > 1 else plan["grid_x"]     # persistent kernels report their tile count in grid_y
+    rows = ctas // (ftiles * max(plan["channel_splits"], 1)) * max(128, plan["tile_rows"] * plan["tile_cols"])
     terms = 1 if L.dtype == "f16" else 3
     return terms * 2.0 * 9 * cp * fp * rows
 

@@ -92,7 +92,7 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
     p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
     p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y; p.tiles_n = pl.tiles_n;
     p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
-    p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit;
+    p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit; p.na = pl.na;
     return p;
 }
 
@@ -390,9 +390,9 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->entries = p.entries;
     } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         const DensePlan &p = h->dense;
-        info->tile_rows = p.TH; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
+        info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
         info->channels_per_stage = 64; info->channel_splits = p.ksplit;
-        info->grid_x = p.grid; info->grid_y = 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
+        info->grid_x = p.grid; info->grid_y = p.halo ? p.n_tiles : 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
         info->entries = static_cast<int64_t>(9) * p.Fp * p.Cp;
     } else {
         info->tile_rows = 1; info->tile_cols = 1; info->filters_per_warp = 1; info->warps_per_cta = 8;

@@ -99,6 +99,8 @@ struct DensePlan {
     int TW = 0, TH = 0, TN = 0; // pixel box (columns, rows, images), TW*TH*TN <= 128
     int tiles_x = 0, tiles_y = 0, tiles_n = 0;
     int box_bytes = 0, stages = 0, smem_bytes = 0, grid = 0;
+    int n_tiles = 0;                       // halo kernel: tiles shared by the persistent CTAs
+    int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
     CUtensorMap mapA{}, mapB{};
 };
@@ -110,7 +112,7 @@ struct DenseParams {
     int N, C, H, W, F;
     int TW, TH, TN, tiles_x, tiles_y, n_ftiles;
     int KB, stages, box_bytes, relu;
-    int tiles_n, iters_per_split, ksplit;
+    int tiles_n, iters_per_split, ksplit, na;
     int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer
     int out_cp;                 // channel pitch of the mode-3 destination
 };

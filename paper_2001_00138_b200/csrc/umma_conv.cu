@@ -38,6 +38,19 @@
 
 namespace patdnn {
 
+#ifdef PATDNN_TRACE
+// Debug-only CTA timeline (build with -DPATDNN_TRACE): 8 time stamps per CTA, read back by patdnn_trace_read().
+__device__ unsigned long long g_trace[1 << 16];
+__device__ __forceinline__ void trace_stamp(int slot) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (blockIdx.x < (1 << 13)) g_trace[blockIdx.x * 8 + slot] = t;
+}
+#define PATDNN_STAMP(slot) trace_stamp(slot)
+#else
+#define PATDNN_STAMP(slot)
+#endif
+
 namespace {
 
 constexpr int kThreads = 192;
@@ -269,11 +282,13 @@ __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__
 // Finish CNT consecutive filters (f_lo ..) of one output pixel: bias + ReLU, then either the caller's NCHW tensor
 // (mode 0) or the next tensor-core layer's split channels-innermost activations (mode 3: [S][N][H][W][out_cp]).
 template <int CNT, typename T>
-__device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT], int f_lo, int n, int y, int x, bool pix_ok) {
+__device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT], const float *s_bias, int f_lo, int n, int y,
+                                           int x, bool pix_ok) {
+    // s_bias: this CTA's bias slice in shared memory, indexed from f_lo (zero beyond the layer's last filter)
 #pragma unroll
     for (int j = 0; j < CNT; ++j) {
         const int f = f_lo + j;
-        float v = (f < p.F) ? a[j] + __ldg(p.bias + f) : 0.f;
+        float v = a[j] + s_bias[j];
         if (p.relu) v = fmaxf(v, 0.f);
         a[j] = (f < p.F) ? v : 0.f;
     }
@@ -327,11 +342,16 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     constexpr int A_BYTES = kTileM * 128;
     constexpr int B_BYTES = BN * 128;
     constexpr int STAGE_BYTES = S * (A_BYTES + B_BYTES);
-    constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    // Narrow filter tiles: the hi and lo weight planes lie back to back in shared memory, so ONE MMA of width 2*BN
+    // forms x_hi*w_hi (columns 0..BN) and x_hi*w_lo (columns BN..2BN); the epilogue adds the two column groups.
+    constexpr bool MERGE = (TERMS == 3) && (BN <= 128);
+    constexpr int ACC_COLS = MERGE ? 2 * BN : BN;
+    constexpr int TMEM_COLS = ACC_COLS < 32 ? 32 : ACC_COLS;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ __align__(8) uint64_t bars[2 * 8 + 1];          // full[stages], empty[stages], accumulator ready
     __shared__ uint32_t tmem_slot;
+    __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = p.stages;
@@ -359,6 +379,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int n = n0 + tn, y = y0 + ty, x = x0 + txx;
     const bool pix_ok = tn < p.TN && n < p.N && y < p.H && x < p.W;
 
+    for (int i = threadIdx.x; i < BN; i += kThreads) s_bias[i] = (f0 + i < p.F) ? p.bias[f0 + i] : 0.f;
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
@@ -393,6 +414,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
+            constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
             bool ok = true;
             for (int it = 0; it < iters && ok; ++it) {
                 const int s = it % stages, use = it / stages;
@@ -405,10 +427,15 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {                   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes
                     const uint64_t koff = static_cast<uint64_t>(2 * k);
-                    umma_f16(tmem_base, a_hi + koff, b_hi + koff, idesc, (it > 0 || k > 0) ? 1u : 0u);
-                    if constexpr (TERMS == 3) {
-                        umma_f16(tmem_base, a_hi + koff, b_lo + koff, idesc, 1u);
+                    if constexpr (MERGE) {
+                        umma_f16(tmem_base, a_hi + koff, b_hi + koff, idesc2, (it > 0 || k > 0) ? 1u : 0u);
                         umma_f16(tmem_base, a_lo + koff, b_hi + koff, idesc, 1u);
+                    } else {
+                        umma_f16(tmem_base, a_hi + koff, b_hi + koff, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                        if constexpr (TERMS == 3) {
+                            umma_f16(tmem_base, a_hi + koff, b_lo + koff, idesc, 1u);
+                            umma_f16(tmem_base, a_lo + koff, b_hi + koff, idesc, 1u);
+                        }
                     }
                 }
                 umma_commit(bar_empty + 8 * s);                 // frees the stage once these MMAs have read it
@@ -427,17 +454,24 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     float a[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) a[j] = __uint_as_float(v[j]);
-                    emit_chunk<32, T>(p, a, f0 + c0, n, y, x, pix_ok);
+                    if constexpr (MERGE) {
+                        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + BN + c0, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) a[j] += __uint_as_float(v[j]);
+                    }
+                    emit_chunk<32, T>(p, a, s_bias + c0, f0 + c0, n, y, x, pix_ok);
                 }
             } else {
                 // partial sums of this K range -> own shared memory, column-major [BN][128] (pipeline buffers are free)
                 float *R = reinterpret_cast<float *>(smem);
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
-                    uint32_t v[32];
+                    uint32_t v[32], v2[32];
                     tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
+                    if constexpr (MERGE) tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + BN + c0, v2);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) R[(c0 + j) * kTileM + m] = __uint_as_float(v[j]);
+                    for (int j = 0; j < 32; ++j)
+                        R[(c0 + j) * kTileM + m] = __uint_as_float(v[j]) + (MERGE ? __uint_as_float(v2[j]) : 0.f);
                 }
             }
         }
@@ -465,13 +499,217 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         a[j] += t;
                     }
                 }
-                emit_chunk<8, T>(p, a, f0 + cbeg + c0, n, y, x, pix_ok);
+                emit_chunk<8, T>(p, a, s_bias + cbeg + c0, f0 + cbeg + c0, n, y, x, pix_ok);
             }
         }
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- halo-sharing, persistent variant for large batches ------------------------------------------------------------
+// The nine taps of a channel block read overlapping pixel windows.  Here a tile is TW x (MT*TH) pixels with TW a
+// multiple of 8 and TW*TH = 128, and per channel block only THREE boxes are loaded -- one per horizontal shift s, each
+// MT*TH+2 rows tall -- instead of nine: one box row is TW*128 bytes, a whole number of 1024-byte swizzle groups, so
+// the operand of vertical tap r is the same buffer entered r rows lower (descriptor start + r*TW*128).
+// CTAs are persistent (one per SM, tiles taken round-robin) and the accumulator is double buffered in TMEM: while the
+// epilogue warps drain tile i, the MMA thread already works on tile i+1.
+// Rings: A (per channel block and shift), B (per channel block and tap), accumulator full/empty (2 buffers).
+template <int BN, int MT, int TERMS, typename T>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
+    constexpr int S = (TERMS == 3) ? 2 : 1;
+    constexpr int B_BYTES = BN * 128;
+    constexpr bool MERGE = (TERMS == 3) && (BN <= 128);          // see conv_umma_kernel: x_hi * [w_hi | w_lo] in one MMA
+    constexpr int ACC_COLS = MERGE ? 2 * BN : BN;
+    constexpr int BUF_COLS = MT * ACC_COLS;                      // one accumulator buffer
+    static_assert(2 * BUF_COLS <= 512, "two accumulator buffers must fit the 512 TMEM columns");
+    constexpr int TMEM_COLS = 2 * BUF_COLS < 32 ? 32 : 2 * BUF_COLS;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) uint64_t bars[4 * 8 + 4];          // fullA, emptyA, fullB, emptyB (8 slots each), acc full/empty x2
+    __shared__ uint32_t tmem_slot;
+    __shared__ float s_bias[2][BN];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NA = p.na, NB = p.stages;
+    const int a_plane = p.box_bytes;                            // one box (one operand plane): (MT*TH+2) * TW * 128 bytes
+    const int a_stage = S * a_plane;
+    const int b_stage = S * B_BYTES;
+    unsigned char *smem_b = smem + NA * a_stage;
+    const uint32_t bar_fa = smem_u32(&bars[0]), bar_ea = smem_u32(&bars[8]), bar_fb = smem_u32(&bars[16]),
+                   bar_eb = smem_u32(&bars[24]), bar_af = smem_u32(&bars[32]), bar_ae = smem_u32(&bars[34]);
+    int *status = p.status;
+    const int row_bytes = p.TW * 128;
+    const int n_tiles = p.n_ftiles * p.tiles_x * p.tiles_y * p.tiles_n;
+    const int KB = p.KB;
+
+    if (threadIdx.x == 0) PATDNN_STAMP(0);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 8; ++s) {
+            mbar_init(bar_fa + 8 * s, 1); mbar_init(bar_ea + 8 * s, 1);
+            mbar_init(bar_fb + 8 * s, 1); mbar_init(bar_eb + 8 * s, 1);
+        }
+        mbar_init(bar_af, 1); mbar_init(bar_af + 8, 1);
+        mbar_init(bar_ae, 4); mbar_init(bar_ae + 8, 4);         // one arrival per epilogue warp
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    if (threadIdx.x == 0) PATDNN_STAMP(1);
+
+    auto decode = [&](int t, int &ft, int &x0, int &y0, int &n) {
+        ft = t % p.n_ftiles; t /= p.n_ftiles;
+        const int tix = t % p.tiles_x; t /= p.tiles_x;
+        const int tiy = t % p.tiles_y; t /= p.tiles_y;
+        n = t; x0 = tix * p.TW; y0 = tiy * (MT * p.TH);
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int ia = 0, ib = 0;                                  // running use counters of the two rings
+            bool ok = true;
+            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                int ft, x0, y0, n;
+                decode(t, ft, x0, y0, n);
+                const int f0 = ft * BN;
+                for (int cb = 0; cb < KB && ok; ++cb) {
+                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                        const int sa = ia % NA, ua = ia / NA;
+                        if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
+                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                        mbar_expect_tx(bar_fa + 8 * sa, S * a_plane);
+#pragma unroll
+                        for (int sp = 0; sp < S; ++sp)
+                            tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - 1, y0 - 1, n, sp);
+                        ++ia;
+                        for (int r = 0; r < 3; ++r) {
+                            const int sb = ib % NB, ub = ib / NB;
+                            if (ub > 0 && !mbar_wait(bar_eb + 8 * sb, (ub - 1) & 1, status, 1)) { ok = false; break; }
+                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            mbar_expect_tx(bar_fb + 8 * sb, S * B_BYTES);
+#pragma unroll
+                            for (int sp = 0; sp < S; ++sp)
+                                tma_load_4d(bbase + sp * B_BYTES, &mapB, bar_fb + 8 * sb, cb * kKBlock, f0, r * 3 + sx, sp);
+                            ++ib;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
+            constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
+            int ia = 0, ib = 0, j = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
+                const int buf = j & 1, ub2 = j >> 1;
+                if (ub2 > 0 && !mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2)) { ok = false; break; }
+                tc_fence_after();
+                bool first = true;
+                for (int cb = 0; cb < KB && ok; ++cb) {
+                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                        const int sa = ia % NA, ua = ia / NA;
+                        ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
+                        if (!ok) break;
+                        if (ia == 0) PATDNN_STAMP(2);
+                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                        for (int r = 0; r < 3 && ok; ++r) {
+                            const int sb = ib % NB, ub = ib / NB;
+                            ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            const uint64_t b_hi = smem_desc_sw128(bbase), b_lo = smem_desc_sw128(bbase + B_BYTES);
+#pragma unroll
+                            for (int mt = 0; mt < MT; ++mt) {
+                                const uint32_t arow = abase + (mt * p.TH + r) * row_bytes;       // 1024-byte aligned
+                                const uint64_t a_hi = smem_desc_sw128(arow), a_lo = smem_desc_sw128(arow + a_plane);
+                                const uint32_t acc = tmem_base + buf * BUF_COLS + mt * ACC_COLS;
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const uint64_t koff = static_cast<uint64_t>(2 * k);
+                                    if constexpr (MERGE) {
+                                        umma_f16(acc, a_hi + koff, b_hi + koff, idesc2, (first && k == 0) ? 0u : 1u);
+                                        umma_f16(acc, a_lo + koff, b_hi + koff, idesc, 1u);
+                                    } else {
+                                        umma_f16(acc, a_hi + koff, b_hi + koff, idesc, (first && k == 0) ? 0u : 1u);
+                                        if constexpr (TERMS == 3) {
+                                            umma_f16(acc, a_hi + koff, b_lo + koff, idesc, 1u);
+                                            umma_f16(acc, a_lo + koff, b_hi + koff, idesc, 1u);
+                                        }
+                                    }
+                                }
+                            }
+                            first = false;
+                            umma_commit(bar_eb + 8 * sb);
+                            ++ib;
+                        }
+                        if (ok) umma_commit(bar_ea + 8 * sa);
+                        ++ia;
+                    }
+                }
+                if (ok) umma_commit(bar_af + 8 * buf);
+            }
+            PATDNN_STAMP(3);
+        }
+    } else {
+        const int q = warp & 3;
+        const int m = q * 32 + lane;
+        const int ty = m / p.TW, txx = m - ty * p.TW;
+        const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
+        int j = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++j) {
+            const int buf = j & 1;
+            int ft, x0, y0, n;
+            decode(t, ft, x0, y0, n);
+            const int f0 = ft * BN;
+            for (int i = et; i < BN; i += 128) s_bias[buf][i] = (f0 + i < p.F) ? p.bias[f0 + i] : 0.f;
+            asm volatile("bar.sync 1, 128;" ::: "memory");     // the four epilogue warps only
+            if (!mbar_wait(bar_af + 8 * buf, (j >> 1) & 1, status, 3)) break;
+            tc_fence_after();
+            if (threadIdx.x == 64 && j == 0) PATDNN_STAMP(4);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const int y = y0 + mt * p.TH + ty, x = x0 + txx;
+                const bool pix_ok = y < p.H && x < p.W;
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t v[32];
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BUF_COLS + mt * ACC_COLS + c0;
+                    tmem_ld32(taddr, v);
+                    float a[32];
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) a[jj] = __uint_as_float(v[jj]);
+                    if constexpr (MERGE) {
+                        tmem_ld32(taddr + BN, v);
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) a[jj] += __uint_as_float(v[jj]);
+                    }
+                    emit_chunk<32, T>(p, a, &s_bias[buf][c0], f0 + c0, n, y, x, pix_ok);
+                }
+            }
+            // this warp is done reading the buffer: hand it back to the MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_ae + 8 * buf) : "memory");
+            if (threadIdx.x == 64 && j == 0) PATDNN_STAMP(5);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) PATDNN_STAMP(6);
     if (warp == 2) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
@@ -496,7 +734,7 @@ EncodeTiledFn encode_fn() {
 template <int BN, int TERMS, typename T>
 cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_kernel<BN, TERMS, T>;
-    if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+    if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
     if (pl.ksplit == 1) {
         kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
         return cudaGetLastError();
@@ -510,7 +748,23 @@ cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t 
     return cudaLaunchKernelEx(&cfg, kern, pl.mapA, pl.mapB, p);
 }
 
+template <int BN, int MT, int TERMS, typename T>
+cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
+    auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T>;
+    if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+    kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
+    return cudaGetLastError();
+}
+
 cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
+    if (pl.halo) {
+#define PATDNN_HALO(bn, mt)                                                                                        \
+    if (pl.BN == bn && pl.MT == mt)                                                                                \
+        return dtype == PATDNN_F16 ? launch_halo<bn, mt, 1, __half>(pl, p, st, prep) : launch_halo<bn, mt, 3, float>(pl, p, st, prep);
+        PATDNN_HALO(256, 1) PATDNN_HALO(128, 1) PATDNN_HALO(64, 1) PATDNN_HALO(64, 2)
+#undef PATDNN_HALO
+        return cudaErrorInvalidConfiguration;
+    }
 #define PATDNN_UMMA(bn)                                                                          \
     if (pl.BN == bn)                                                                             \
         return dtype == PATDNN_F16 ? launch_umma<bn, 1, __half>(pl, p, st, prep) : launch_umma<bn, 3, float>(pl, p, st, prep);
@@ -545,17 +799,17 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
         if (score > best) { best = score; pl.TW = tw; pl.TH = th; pl.TN = tn; pl.tiles_x = (int)tx; pl.tiles_y = (int)ty; pl.tiles_n = (int)tz; }
     }
     // Few pixel tiles (small batch): cut the K loop into ks ranges, one CTA each, ks CTAs forming a cluster that sums
-    // its partial tiles through distributed shared memory; only when even 8 ranges leave most SMs idle, narrow the
-    // filter tile as well (a wide tile makes every loaded activation byte feed more MMA work).
+    // its partial tiles through distributed shared memory (measured: 4 ranges beat 8, whose reduction and cluster
+    // scheduling cost more than the shorter loop saves); if that still leaves most SMs idle, narrow the filter tile.
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
     const int total_iters = 9 * pl.KB;
-    while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 8 < 120) pl.BN /= 2;
+    while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 4 < 100) pl.BN /= 2;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
     int ks = 1;
     if (base_grid < 100)
-        while (ks < 8 && base_grid * ks * 2 <= 296 && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
+        while (ks < 4 && base_grid * ks * 2 <= 296 && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
     if (const char *ov = std::getenv("PATDNN_KSPLIT")) {
         const int want = atoi(ov);
         if ((want == 1 || want == 2 || want == 4 || want == 8) && want <= total_iters && pl.BN / want >= 8) ks = want;
@@ -567,6 +821,42 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
     pl.smem_bytes = pl.stages * stage + 1024;
     pl.grid = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles * pl.ksplit;
+
+    // Large grids: the halo-sharing kernel (three boxes per channel block instead of nine) if a TW x TH = 128 box
+    // with TW a multiple of 8 wastes no more pixels than the free-form box does.
+    const char *hv = std::getenv("PATDNN_HALO");
+    if (pl.ksplit == 1 && pl.BN >= 64 && !(hv && hv[0] == '0')) {
+        const double util_now = static_cast<double>(N) * H * W / (static_cast<double>(ptiles) * kTileM);
+        int btw = 0; double butil = 0;
+        for (int tw : {32, 16, 8, 64, 128}) {                      // ties: 32-wide boxes first (128-byte store rows, 1.5x halo)
+            const int th = kTileM / tw;
+            const double u = static_cast<double>(H) * W /
+                             (static_cast<double>((W + tw - 1) / tw) * tw * static_cast<double>((H + th - 1) / th) * th);
+            const int mt_try = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
+            const bool fits = 2 * pl.S * (mt_try * th + 2) * tw * 128 + 2 * pl.S * pl.BN * 128 <= 218 * 1024;
+            if (fits && u > butil + 1e-9) { butil = u; btw = tw; }
+        }
+        if (btw && butil >= util_now - 0.02) {
+            const int th = kTileM / btw;
+            int mt = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
+            if (const char *mv = std::getenv("PATDNN_MT")) mt = (atoi(mv) == 2 && pl.BN == 64) ? 2 : 1;
+            const int a_stage = pl.S * (mt * th + 2) * btw * 128;
+            const int b_stage = pl.S * pl.BN * 128;
+            int na = 2, nb = 2;
+            const int budget = 218 * 1024;
+            while (nb < 6 && na * a_stage + (nb + 1) * b_stage <= budget) ++nb;
+            if (na * a_stage + nb * b_stage <= budget) {
+                while (na < 3 && (na + 1) * a_stage + nb * b_stage <= budget) ++na;
+                pl.halo = 1; pl.MT = mt; pl.TW = btw; pl.TH = th; pl.TN = 1;
+                pl.tiles_x = (W + btw - 1) / btw; pl.tiles_y = (H + mt * th - 1) / (mt * th); pl.tiles_n = N;
+                pl.box_bytes = (mt * th + 2) * btw * 128;
+                pl.na = na; pl.stages = nb;
+                pl.smem_bytes = na * a_stage + nb * b_stage + 1024;
+                pl.n_tiles = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
+                pl.grid = std::min(pl.n_tiles, 148);             // persistent CTAs, one per SM
+            }
+        }
+    }
 }
 
 // Dense split weights [S][9][Fp][Cp] (16-bit words) from the canonical FKW arrays.
@@ -606,7 +896,8 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
         cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)pl.S};
         cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)W * pl.Cp * 2, (cuuint64_t)H * W * pl.Cp * 2,
                                  (cuuint64_t)N * H * W * pl.Cp * 2};
-        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)pl.TH, (cuuint32_t)pl.TN, 1};
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)(pl.halo ? pl.MT * pl.TH + 2 : pl.TH),
+                             (cuuint32_t)pl.TN, 1};
         cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (enc(&pl.mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -645,6 +936,12 @@ int static_scratch_address(void **ptr) {
     *ptr = addr[dev];
     return PATDNN_OK;
 }
+
+#ifdef PATDNN_TRACE
+extern "C" __attribute__((visibility("default"))) int patdnn_trace_read(unsigned long long *host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(unsigned long long) * n);
+}
+#endif
 
 cudaError_t prepare_dense(const DensePlan &pl, int dtype) {
     DenseParams dummy{};
