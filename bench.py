@@ -100,14 +100,15 @@ def executed_tensor_flops(L, plan):
     """16-bit MMA flops the dense tensor-core kernel issues for a layer (0 for the CUDA-core kernels)."""
     if plan["variant"] != 4:
         return 0.0
-    cp = (L.C + 63) // 64 * 64
+    taps = 1 if 9 * L.C <= 64 else 9          # tiny C: neighbourhood gathered into the channel dimension
+    cp = 64 if taps == 1 else (L.C + 63) // 64 * 64
     bn = plan["filters_per_warp"]
     fp = (L.F + bn - 1) // bn * bn
     ftiles = fp // bn
     ctas = plan["grid_y"] if plan["grid_y"] > 1 else plan["grid_x"]     # persistent kernels report their tile count in grid_y
     rows = ctas // (ftiles * max(plan["channel_splits"], 1)) * max(128, plan["tile_rows"] * plan["tile_cols"])
     terms = 1 if L.dtype == "f16" else 3
-    return terms * 2.0 * 9 * cp * fp * rows
+    return terms * 2.0 * taps * cp * fp * rows
 
 
 class VggStack:

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -92,7 +93,7 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
     p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F;
     p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y; p.tiles_n = pl.tiles_n;
     p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
-    p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit; p.na = pl.na;
+    p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit; p.na = pl.na; p.taps = pl.taps;
     return p;
 }
 
@@ -106,6 +107,9 @@ static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const pat
     } else {
         p.mode = 0; p.out = out;
     }
+#ifdef PATDNN_TRACE
+    if (std::getenv("PATDNN_NOSTORE")) p.mode = 9;
+#endif
     cudaError_t e = launch_dense_gemm(pl, p, h->desc.dtype, st);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core kernel launch");
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -115,7 +119,8 @@ static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const pat
 // One tensor-core layer from an NCHW input to its finished NCHW output.
 static int dense_forward(patdnn_layer *h, const DensePlan &pl, const void *in, void *act, void *out, cudaStream_t st) {
     const patdnn_desc &d = h->desc;
-    cudaError_t e = launch_transition(in, d.dtype == PATDNN_F16, act, nullptr, 0, 0, 0, d.N, d.C, d.H, d.W, pl.Cp, pl.S, st);
+    cudaError_t e = pl.im2col ? launch_im2col(in, d.dtype == PATDNN_F16, act, d.N, d.C, d.H, d.W, pl.S, st)
+                              : launch_transition(in, d.dtype == PATDNN_F16, act, nullptr, 0, 0, 0, d.N, d.C, d.H, d.W, pl.Cp, pl.S, st);
     if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return dense_gemm(h, pl, out, nullptr, st);
@@ -157,11 +162,13 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                     plan_dense(desc->F, desc->C, desc->N, desc->H, desc->W, desc->dtype, dp);
                     const double terms = desc->dtype == PATDNN_F16 ? 1.0 : 3.0;
                     const double rows = static_cast<double>(dp.tiles_x) * dp.tiles_y * dp.tiles_n * 128.0;
-                    const double t_dense = terms * 2.0 * 9.0 * dp.Cp * dp.Fp * rows / 9.0e14 +
+                    const double t_dense = terms * 2.0 * dp.taps * dp.Cp * dp.Fp * rows / 9.0e14 +
                                            static_cast<double>(desc->N) * desc->H * desc->W * (desc->C * 4.0 + dp.Cp * 2.0 * dp.S) / 4.0e12 +
                                            4e-6;
                     const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / 1.2e13 + 4e-6;
-                    if (t_dense < t_tiled) h->variant = PATDNN_VARIANT_DENSE_TC;
+                    // layers with 9*C <= 64 (gathered-neighbourhood GEMM) are store-bound there: measured slower than the
+                    // CUDA-core kernel on the RGB first layer, so AUTO leaves them on it unless it cannot run the layer
+                    if (t_dense < t_tiled && (!dp.im2col || !can_tile)) h->variant = PATDNN_VARIANT_DENSE_TC;
                 }
             } else {
                 h->variant = desc->variant;
@@ -393,7 +400,7 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
         info->channels_per_stage = 64; info->channel_splits = p.ksplit;
         info->grid_x = p.grid; info->grid_y = p.halo ? p.n_tiles : 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
-        info->entries = static_cast<int64_t>(9) * p.Fp * p.Cp;
+        info->entries = static_cast<int64_t>(p.taps) * p.Fp * p.Cp;
     } else {
         info->tile_rows = 1; info->tile_cols = 1; info->filters_per_warp = 1; info->warps_per_cta = 8;
         info->channels_per_stage = 0; info->channel_splits = 1;
@@ -470,13 +477,24 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
         const bool last = (i == n - 1);
         const bool is_dense = h->variant == PATDNN_VARIANT_DENSE_TC;
         if (is_dense) {
-            if (!direct) {
+            if (!direct && h->dense.im2col) {
+                if (cur_pool) {
+                    const int rc = patdnn_maxpool2x2(cur, s->buf[which], d.N, d.C, curH, curW, d.dtype, stream);
+                    if (rc) return rc;
+                    cur = s->buf[which];
+                    which ^= 1;
+                }
+                cudaError_t e = launch_im2col(cur, d.dtype == PATDNN_F16, h->d_act, d.N, d.C, d.H, d.W, h->dense.S, st);
+                if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
+                g_launches.fetch_add(1, std::memory_order_relaxed);
+            } else if (!direct) {
                 cudaError_t e = launch_transition(cur, d.dtype == PATDNN_F16, h->d_act, nullptr, 0, cur_pool, 0, d.N, d.C,
                                                   curH, curW, h->dense.Cp, h->dense.S, st);
                 if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
-            patdnn_layer *next = (!last && !s->pool[i] && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC)
+            patdnn_layer *next = (!last && !s->pool[i] && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC &&
+                                  !s->layers[i + 1]->dense.im2col)
                                      ? s->layers[i + 1] : nullptr;
             void *dst = next ? nullptr : ((last && !s->pool[i]) ? out : s->buf[which]);
             const int rc = dense_gemm(h, h->dense, dst, next, st);

@@ -99,6 +99,7 @@ struct DensePlan {
     int TW = 0, TH = 0, TN = 0; // pixel box (columns, rows, images), TW*TH*TN <= 128
     int tiles_x = 0, tiles_y = 0, tiles_n = 0;
     int box_bytes = 0, stages = 0, smem_bytes = 0, grid = 0;
+    int im2col = 0, taps = 9;              // tiny C: 3x3 neighbourhood gathered into the channel dimension (one tap)
     int n_tiles = 0;                       // halo kernel: tiles shared by the persistent CTAs
     int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
@@ -112,7 +113,7 @@ struct DenseParams {
     int N, C, H, W, F;
     int TW, TH, TN, tiles_x, tiles_y, n_ftiles;
     int KB, stages, box_bytes, relu;
-    int tiles_n, iters_per_split, ksplit, na;
+    int tiles_n, iters_per_split, ksplit, na, taps;
     int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer
     int out_cp;                 // channel pitch of the mode-3 destination
 };
@@ -127,6 +128,7 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
 cudaError_t prepare_dense(const DensePlan &pl, int dtype);
 cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const float *bias, int relu, int pool, int clear,
                               int N, int C, int Hs, int Ws, int Cp, int S, cudaStream_t st);
+cudaError_t launch_im2col(const void *src, int src_is_half, void *dst, int N, int C, int H, int W, int S, cudaStream_t st);
 cudaError_t launch_dense_gemm(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st);
 
 }  // namespace patdnn

@@ -54,6 +54,7 @@ __device__ __forceinline__ void trace_stamp(int slot) {
 namespace {
 
 constexpr int kThreads = 192;
+constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kTileM = 128;
 constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
 constexpr uint32_t kSpinLimit = 1u << 21;    // bounded mbarrier polling: each poll may block up to ~1 us (hint below)
@@ -279,6 +280,58 @@ __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__
     }
 }
 
+// Layers with very few input channels (9*C <= 64, e.g. an RGB first layer): gather the 3x3 neighbourhood into the
+// channel dimension, k = 9*c + tap, so that the whole layer is ONE 64-deep GEMM step instead of nine mostly-padding ones.
+// dst is [S][N][H][W][64].  A block stages the three input rows of a 32-pixel row segment for all channels in shared
+// memory; then 8 threads per pixel each build 8 consecutive k and store 16 bytes per operand plane.
+// grid = (ceil(W/32), H, N), block = 256.
+template <typename T>
+__global__ void __launch_bounds__(256) im2col_kernel(const T *__restrict__ src, uint16_t *__restrict__ dst, int N, int C,
+                                                      int H, int W, int S) {
+    __shared__ float rows[7][3][36];                             // [channel][row -1..1][column -1..32 (+pad)]
+    const int x0 = blockIdx.x * 32, y = blockIdx.y, n = blockIdx.z;
+    for (int i = threadIdx.x; i < C * 3 * 34; i += 256) {
+        const int c = i / 102, rem = i - c * 102, r = rem / 34, j = rem - r * 34;
+        const int yy = y + r - 1, xx = x0 + j - 1;
+        float v = 0.f;
+        if (yy >= 0 && yy < H && xx >= 0 && xx < W) {
+            const T raw = src[((static_cast<size_t>(n) * C + c) * H + yy) * W + xx];
+            if constexpr (sizeof(T) == 2) v = __half2float(raw); else v = raw;
+        }
+        rows[c][r][j] = v;
+    }
+    __syncthreads();
+    const int px = threadIdx.x >> 3, part = threadIdx.x & 7;
+    const int x = x0 + px;
+    if (x >= W) return;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        float v[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int k = 8 * part + 2 * e + h;
+            const int c = k / 9, t = k - 9 * c;
+            v[h] = (c < C) ? rows[c][t / 3][px + t % 3] : 0.f;
+        }
+        if (S == 2) {
+            const __nv_bfloat16 ah = __float2bfloat16_rn(v[0]), bh = __float2bfloat16_rn(v[1]);
+            const __nv_bfloat16 al = __float2bfloat16_rn(v[0] - __bfloat162float(ah));
+            const __nv_bfloat16 bl = __float2bfloat16_rn(v[1] - __bfloat162float(bh));
+            hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
+            lo[e] = static_cast<uint32_t>(__bfloat16_as_ushort(al)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
+        } else {
+            hi[e] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v[0]))) |
+                    (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v[1]))) << 16);
+        }
+    }
+    const size_t pix = (static_cast<size_t>(n) * H + y) * W + x;
+    const size_t o = pix * 64 + 8 * part;
+    *reinterpret_cast<uint4 *>(dst + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    if (S == 2)
+        *reinterpret_cast<uint4 *>(dst + static_cast<size_t>(N) * H * W * 64 + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+
 // Finish CNT consecutive filters (f_lo ..) of one output pixel: bias + ReLU, then either the caller's NCHW tensor
 // (mode 0) or the next tensor-core layer's split channels-innermost activations (mode 3: [S][N][H][W][out_cp]).
 template <int CNT, typename T>
@@ -293,6 +346,9 @@ __device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT]
         a[j] = (f < p.F) ? v : 0.f;
     }
     if (!pix_ok) return;
+#ifdef PATDNN_TRACE
+    if (p.mode == 9) { if (a[0] == 1.2345e-30f) static_cast<float *>(p.out)[0] = a[1]; return; }   // timing probe: no stores
+#endif
     if (p.mode == 0) {
         T *out = static_cast<T *>(p.out);
         const size_t plane = static_cast<size_t>(p.H) * p.W;
@@ -368,8 +424,9 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int tiy = pt % p.tiles_y; pt /= p.tiles_y;
     const int tin = pt;
     const int x0 = tix * p.TW, y0 = tiy * p.TH, n0 = tin * p.TN, f0 = ft * BN;
-    const int it0 = rank * (9 * p.KB) / ks;                     // even split: every range holds at least one iteration
-    const int iters = (rank + 1) * (9 * p.KB) / ks - it0;
+    const int total_iters = p.taps * p.KB;                      // taps = 9, or 1 for gathered (im2col) activations
+    const int it0 = rank * total_iters / ks;                    // even split: every range holds at least one iteration
+    const int iters = (rank + 1) * total_iters / ks - it0;
     // output pixel of this thread when it acts as an epilogue thread (warps 2..5 cover the 128 accumulator rows)
     const int q = warp & 3;
     const int m = q * 32 + lane;
@@ -400,8 +457,8 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             for (int it = 0; it < iters; ++it) {
                 const int s = it % stages, use = it / stages;
                 if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1, status, 1)) break;
-                const int cb = (it0 + it) / 9, tap = (it0 + it) - cb * 9;
-                const int r = tap / 3, sx = tap - 3 * r;
+                const int cb = (it0 + it) / p.taps, tap = (it0 + it) - cb * p.taps;
+                const int r = p.taps == 9 ? tap / 3 : 1, sx = p.taps == 9 ? tap - 3 * r : 1;
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
                 mbar_expect_tx(bar_full + 8 * s, tx_bytes);
 #pragma unroll
@@ -520,7 +577,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // epilogue warps drain tile i, the MMA thread already works on tile i+1.
 // Rings: A (per channel block and shift), B (per channel block and tap), accumulator full/empty (2 buffers).
 template <int BN, int MT, int TERMS, typename T>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kHaloThreads, 1)
 conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
     constexpr int S = (TERMS == 3) ? 2 : 1;
     constexpr int B_BYTES = BN * 128;
@@ -547,6 +604,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     const int row_bytes = p.TW * 128;
     const int n_tiles = p.n_ftiles * p.tiles_x * p.tiles_y * p.tiles_n;
     const int KB = p.KB;
+    const int nshift = p.taps == 9 ? 3 : 1;                     // 3 horizontal shifts x 3 vertical taps, or one gathered tap
 
     if (threadIdx.x == 0) PATDNN_STAMP(0);
     if (threadIdx.x == 0) {
@@ -555,7 +613,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             mbar_init(bar_fb + 8 * s, 1); mbar_init(bar_eb + 8 * s, 1);
         }
         mbar_init(bar_af, 1); mbar_init(bar_af + 8, 1);
-        mbar_init(bar_ae, 4); mbar_init(bar_ae + 8, 4);         // one arrival per epilogue warp
+        mbar_init(bar_ae, 8); mbar_init(bar_ae + 8, 8);         // one arrival per epilogue warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 2) {
@@ -584,23 +642,23 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 decode(t, ft, x0, y0, n);
                 const int f0 = ft * BN;
                 for (int cb = 0; cb < KB && ok; ++cb) {
-                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                    for (int sx = 0; sx < nshift && ok; ++sx) {
                         const int sa = ia % NA, ua = ia / NA;
                         if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
                         const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
                         mbar_expect_tx(bar_fa + 8 * sa, S * a_plane);
 #pragma unroll
                         for (int sp = 0; sp < S; ++sp)
-                            tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - 1, y0 - 1, n, sp);
+                            tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - (nshift >> 1), y0 - (nshift >> 1), n, sp);
                         ++ia;
-                        for (int r = 0; r < 3; ++r) {
+                        for (int r = 0; r < nshift; ++r) {
                             const int sb = ib % NB, ub = ib / NB;
                             if (ub > 0 && !mbar_wait(bar_eb + 8 * sb, (ub - 1) & 1, status, 1)) { ok = false; break; }
                             const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
                             mbar_expect_tx(bar_fb + 8 * sb, S * B_BYTES);
 #pragma unroll
                             for (int sp = 0; sp < S; ++sp)
-                                tma_load_4d(bbase + sp * B_BYTES, &mapB, bar_fb + 8 * sb, cb * kKBlock, f0, r * 3 + sx, sp);
+                                tma_load_4d(bbase + sp * B_BYTES, &mapB, bar_fb + 8 * sb, cb * kKBlock, f0, r * nshift + sx, sp);
                             ++ib;
                         }
                     }
@@ -619,13 +677,13 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 tc_fence_after();
                 bool first = true;
                 for (int cb = 0; cb < KB && ok; ++cb) {
-                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                    for (int sx = 0; sx < nshift && ok; ++sx) {
                         const int sa = ia % NA, ua = ia / NA;
                         ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
                         if (!ok) break;
                         if (ia == 0) PATDNN_STAMP(2);
                         const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
-                        for (int r = 0; r < 3 && ok; ++r) {
+                        for (int r = 0; r < nshift && ok; ++r) {
                             const int sb = ib % NB, ub = ib / NB;
                             ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
                             if (!ok) break;
@@ -665,18 +723,20 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             PATDNN_STAMP(3);
         }
     } else {
+        // eight epilogue warps: warp w reads TMEM lanes 32*(w%4).. and one half of the filter columns
         const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int m = q * 32 + lane;
         const int ty = m / p.TW, txx = m - ty * p.TW;
-        const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
+        const int et = threadIdx.x - 64;                         // 0..255 among the epilogue threads
         int j = 0;
         for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++j) {
             const int buf = j & 1;
             int ft, x0, y0, n;
             decode(t, ft, x0, y0, n);
             const int f0 = ft * BN;
-            for (int i = et; i < BN; i += 128) s_bias[buf][i] = (f0 + i < p.F) ? p.bias[f0 + i] : 0.f;
-            asm volatile("bar.sync 1, 128;" ::: "memory");     // the four epilogue warps only
+            for (int i = et; i < BN; i += 256) s_bias[buf][i] = (f0 + i < p.F) ? p.bias[f0 + i] : 0.f;
+            asm volatile("bar.sync 1, 256;" ::: "memory");     // the eight epilogue warps only
             if (!mbar_wait(bar_af + 8 * buf, (j >> 1) & 1, status, 3)) break;
             tc_fence_after();
             if (threadIdx.x == 64 && j == 0) PATDNN_STAMP(4);
@@ -685,7 +745,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 const int y = y0 + mt * p.TH + ty, x = x0 + txx;
                 const bool pix_ok = y < p.H && x < p.W;
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
                     uint32_t v[32];
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BUF_COLS + mt * ACC_COLS + c0;
                     tmem_ld32(taddr, v);
@@ -752,7 +812,7 @@ template <int BN, int MT, int TERMS, typename T>
 cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-    kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
+    kern<<<pl.grid, kHaloThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
     return cudaGetLastError();
 }
 
@@ -783,7 +843,9 @@ bool dense_supported(int F, int C, int N, int H, int W) {
 void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     pl = DensePlan();
     pl.S = dtype == PATDNN_F16 ? 1 : 2;
-    pl.Cp = (C + kKBlock - 1) / kKBlock * kKBlock;
+    pl.im2col = (9 * C <= kKBlock) ? 1 : 0;                        // tiny C: taps gathered into the channel dimension
+    pl.taps = pl.im2col ? 1 : 9;
+    pl.Cp = pl.im2col ? kKBlock : (C + kKBlock - 1) / kKBlock * kKBlock;
     pl.KB = pl.Cp / kKBlock;
     pl.BN = F > 128 ? 256 : (F > 64 ? 128 : (F > 32 ? 64 : 32));
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
@@ -802,7 +864,7 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     // its partial tiles through distributed shared memory (measured: 4 ranges beat 8, whose reduction and cluster
     // scheduling cost more than the shorter loop saves); if that still leaves most SMs idle, narrow the filter tile.
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
-    const int total_iters = 9 * pl.KB;
+    const int total_iters = pl.taps * pl.KB;
     while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 4 < 100) pl.BN /= 2;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
@@ -833,14 +895,16 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
             const double u = static_cast<double>(H) * W /
                              (static_cast<double>((W + tw - 1) / tw) * tw * static_cast<double>((H + th - 1) / th) * th);
             const int mt_try = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
-            const bool fits = 2 * pl.S * (mt_try * th + 2) * tw * 128 + 2 * pl.S * pl.BN * 128 <= 218 * 1024;
+            const int hr = pl.im2col ? 0 : 2;                       // halo rows
+            const bool fits = 2 * pl.S * (mt_try * th + hr) * tw * 128 + 2 * pl.S * pl.BN * 128 <= 218 * 1024;
             if (fits && u > butil + 1e-9) { butil = u; btw = tw; }
         }
         if (btw && butil >= util_now - 0.02) {
             const int th = kTileM / btw;
             int mt = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
             if (const char *mv = std::getenv("PATDNN_MT")) mt = (atoi(mv) == 2 && pl.BN == 64) ? 2 : 1;
-            const int a_stage = pl.S * (mt * th + 2) * btw * 128;
+            const int hr = pl.im2col ? 0 : 2;
+            const int a_stage = pl.S * (mt * th + hr) * btw * 128;
             const int b_stage = pl.S * pl.BN * 128;
             int na = 2, nb = 2;
             const int budget = 218 * 1024;
@@ -849,7 +913,7 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
                 while (na < 3 && (na + 1) * a_stage + nb * b_stage <= budget) ++na;
                 pl.halo = 1; pl.MT = mt; pl.TW = btw; pl.TH = th; pl.TN = 1;
                 pl.tiles_x = (W + btw - 1) / btw; pl.tiles_y = (H + mt * th - 1) / (mt * th); pl.tiles_n = N;
-                pl.box_bytes = (mt * th + 2) * btw * 128;
+                pl.box_bytes = (mt * th + hr) * btw * 128;
                 pl.na = na; pl.stages = nb;
                 pl.smem_bytes = na * a_stage + nb * b_stage + 1024;
                 pl.n_tiles = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
@@ -861,7 +925,7 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
 
 // Dense split weights [S][9][Fp][Cp] (16-bit words) from the canonical FKW arrays.
 void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16_t> &w) {
-    const size_t plane = static_cast<size_t>(9) * pl.Fp * pl.Cp;
+    const size_t plane = static_cast<size_t>(pl.taps) * pl.Fp * pl.Cp;
     w.assign(plane * pl.S, 0);
     for (int i = 0; i < fkw.F; ++i) {
         const int f = fkw.reorder[i];
@@ -872,7 +936,8 @@ void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16
             for (int t = 0; t < 9; ++t) {
                 if (!((mask >> t) & 1u)) continue;
                 const float v = fkw.weight_f32[static_cast<size_t>(k) * 4 + j++];
-                const size_t o = (static_cast<size_t>(t) * pl.Fp + f) * pl.Cp + c;
+                const size_t o = pl.im2col ? static_cast<size_t>(f) * pl.Cp + 9 * c + t
+                                           : (static_cast<size_t>(t) * pl.Fp + f) * pl.Cp + c;
                 if (pl.S == 2) {
                     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
                     const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
@@ -896,7 +961,7 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
         cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)pl.S};
         cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)W * pl.Cp * 2, (cuuint64_t)H * W * pl.Cp * 2,
                                  (cuuint64_t)N * H * W * pl.Cp * 2};
-        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)(pl.halo ? pl.MT * pl.TH + 2 : pl.TH),
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)(pl.halo ? pl.MT * pl.TH + (pl.im2col ? 0 : 2) : pl.TH),
                              (cuuint32_t)pl.TN, 1};
         cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (enc(&pl.mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -904,8 +969,8 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
             return PATDNN_E_CUDA;
     }
     {
-        cuuint64_t dims[4] = {(cuuint64_t)pl.Cp, (cuuint64_t)pl.Fp, 9, (cuuint64_t)pl.S};
-        cuuint64_t strides[3] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)pl.Fp * pl.Cp * 2, (cuuint64_t)9 * pl.Fp * pl.Cp * 2};
+        cuuint64_t dims[4] = {(cuuint64_t)pl.Cp, (cuuint64_t)pl.Fp, (cuuint64_t)pl.taps, (cuuint64_t)pl.S};
+        cuuint64_t strides[3] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)pl.Fp * pl.Cp * 2, (cuuint64_t)pl.taps * pl.Fp * pl.Cp * 2};
         cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.BN, 1, 1};
         cuuint32_t es[4] = {1, 1, 1, 1};
         if (enc(&pl.mapB, dt, 4, d_w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -970,6 +1035,16 @@ cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const
     else
         transition_kernel<float><<<grid, block, 0, st>>>(static_cast<float *>(const_cast<void *>(src)),
                                                          static_cast<uint16_t *>(dst), bias, relu, pool, clear, N, C, Hs, Ws, Cp, S);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_im2col(const void *src, int src_is_half, void *dst, int N, int C, int H, int W, int S, cudaStream_t st) {
+    if (N == 0) return cudaSuccess;
+    dim3 grid((W + 31) / 32, H, N);
+    if (src_is_half)
+        im2col_kernel<__half><<<grid, 256, 0, st>>>(static_cast<const __half *>(src), static_cast<uint16_t *>(dst), N, C, H, W, S);
+    else
+        im2col_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(src), static_cast<uint16_t *>(dst), N, C, H, W, S);
     return cudaGetLastError();
 }
 
