@@ -29,9 +29,10 @@ if ROOT not in sys.path:
 
 SM_COUNT, FP32_LANES, SM_MAX_GHZ = 148, 128, 1.965
 ALU_PEAK_TFLOPS = SM_COUNT * FP32_LANES * 2 * SM_MAX_GHZ / 1e3     # 74.45: FP32 FMA lanes x 2 flop x max SM clock
-# dram__bytes_read.sum + dram__bytes_write.sum of one conv_umma_kernel launch, from the ncu capture summarised under
-# profiles/ (None until a capture of the benchmark's layer shape exists)
-TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (conv_umma_halo_kernel on the
+# 256 -> 256 @ 56x56 layer): 28.5 MB in the ncu capture at batch 8 (profiles/conv_umma_halo_kernel_vgg16_L06_n8.txt),
+# scaled by the units of a batch-32 launch (x4; reads grow in proportion, the output additionally leaves L2 at that size)
+TRAFFIC_BYTES_PER_LAUNCH = 4 * (28109312 + 387328)
 
 
 def measured_peaks():
@@ -54,7 +55,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -185,7 +186,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=32)
@@ -339,8 +340,9 @@ def main():
         "roofline": {"bound": "tensor", "achieved": tc_ach, "peak": tc_peak, "unit": "TFLOP/s",
                      "frac": tc_ach / tc_peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
                      "peak_source": f"{peak_kind} bf16 cuBLAS peak (sustained, kernel timed inside a long step)",
-                     "kernel": "conv_umma_kernel (tcgen05 implicit GEMM, bf16 hi/lo split, 3 MMAs per product); "
-                               "achieved = executed 16-bit MMA flops / summed launch time (layout kernel included)",
+                     "kernel": "conv_umma_halo_kernel / conv_umma_kernel (tcgen05 implicit GEMM, bf16 hi/lo split, three "
+                               "products per fp32 product); achieved = executed 16-bit MMA flops / summed launch time of "
+                               "the tensor-core layers (layout kernels included)",
                      "launches_per_step": sum(1 for f, _ in tc if f > 0), "us_per_step": tc_us},
         "north_star_roofline": {"definition": "per layer max(2*nonzero MACs / FP32 CUDA-core peak, algorithmic bytes / "
                                               "measured HBM bandwidth); stack fraction = sum roofline / sum conv time",
@@ -348,6 +350,9 @@ def main():
                                 "peak_source": "148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
                                 "frac": achieved / ALU_PEAK_TFLOPS, "stack_roofline_us": roof_us,
                                 "stack_conv_us": conv_us, "stack_frac": roof_us / conv_us,
+                                "stack_frac_step": roof_us / (ms * 1e3),
+                                "note": "stack_frac uses the sum of per-layer launch times (each layer run alone, NCHW in "
+                                        "and out); stack_frac_step uses the timed step of the chained stack, pools included",
                                 "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
         "layers": [{"name": n, "us": round(u, 2), "roofline_us": round(c[2], 2), "bound": c[3],
                     "frac": round(c[2] / u, 3), "kernel": {3: "tiled", 4: "dense_tc"}.get(p["variant"], "generic"),
@@ -362,6 +367,7 @@ def main():
                           "value": r1["flops"] / (r1["ms_per_step"] * 1e-3) / 1e9, "unit": "GFLOP/s",
                           "l2": "256 MB buffer written between timed steps", "stack_conv_us": conv1,
                           "stack_roofline_us": roof1, "stack_frac": roof1 / conv1,
+                          "stack_frac_step": roof1 / (r1["ms_per_step"] * 1e3),
                           "layer_us": [round(u, 2) for u in r1["layer_us"]],
                           "e2e_ms": r1["e2e_ms"]}
         import oracle

@@ -848,6 +848,10 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     pl.Cp = pl.im2col ? kKBlock : (C + kKBlock - 1) / kKBlock * kKBlock;
     pl.KB = pl.Cp / kKBlock;
     pl.BN = F > 128 ? 256 : (F > 64 ? 128 : (F > 32 ? 64 : 32));
+    if (const char *bv = std::getenv("PATDNN_BN")) {             // tuning override
+        const int want = atoi(bv);
+        if (want == 32 || want == 64 || want == 128 || want == 256) pl.BN = std::min(pl.BN, want);
+    }
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     double best = -1;
