@@ -154,6 +154,88 @@ def time_oracle_sample(synth, seconds_hint=15.0):
                                          f"{dt * 1e3:.1f} ms each, OpenMP over filters"}
 
 
+def time_layer(h, x, y, stream, torch, reps=20, flush=None):
+    """Mean launch time (us) of one layer call, CUDA events on the launching stream."""
+    for _ in range(3):
+        h.conv(x, y, stream)
+    torch.cuda.synchronize()
+    tot = 0.0
+    for _ in range(reps):
+        if flush is not None:
+            flush.fill_(1.0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        h.conv(x, y, stream)
+        b.record()
+        torch.cuda.synchronize()
+        tot += a.elapsed_time(b)
+    return tot / reps * 1e3
+
+
+def run_suite(args):
+    """The other configurations of the baseline as a table (one JSON object per line on stdout):
+    config 2, the ResNet-50-shaped fp16 layers, the pattern-count x connectivity sweep (with the filter reorder on and
+    with a seeded random filter order), and the ablation ladder no-opt -> +reorder -> tiled -> tensor cores."""
+    import torch
+    from paper_2001_00138_b200 import build as lib_build, binding as B, synth
+    lib_build.build_library()
+    B.load()
+    peaks, _ = measured_peaks()
+    hbm = float(peaks["hbm_gbs"])
+    stream = torch.cuda.current_stream().cuda_stream
+    flush = torch.empty(256 * 1024 * 1024 // 4, device="cuda")
+    variants = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense_tc": 4}
+
+    def measure(tag, L, N, variant="auto", order=None, reps=20):
+        dt = B.F16 if L.dtype == "f16" else B.F32
+        tdt = torch.float16 if L.dtype == "f16" else torch.float32
+        try:
+            h = B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, dtype=dt, relu=True, bias=L.bias,
+                         order=order, variant=variants[variant])
+        except B.PatdnnError as e:
+            print(json.dumps({"suite": tag, "layer": L.name, "batch": N, "variant": variant, "error": str(e)}))
+            return
+        x = torch.rand((N, L.C, L.H, L.W), device="cuda").to(tdt)
+        y = torch.empty((N, L.F, L.H, L.W), device="cuda", dtype=tdt)
+        small = x.numel() * x.element_size() + y.numel() * y.element_size() < 128 * 2**20
+        us = time_layer(h, x, y, stream, torch, reps=reps, flush=flush if small else None)
+        L.N = N
+        flops, byts, roof_us, bound = layer_costs(L, hbm)
+        plan = h.plan()
+        print(json.dumps({"suite": tag, "layer": L.name, "batch": N, "variant": variant,
+                          "kernel": {1: "noopt", 2: "reorder", 3: "tiled", 4: "dense_tc"}[plan["variant"]],
+                          "filter_order": "random" if order is not None else "fkr", "K": L.K,
+                          "us": round(us, 2), "gflops_nonzero": round(flops / us / 1e3, 1),
+                          "roofline_us": round(roof_us, 2), "bound": bound, "frac": round(roof_us / us, 3),
+                          "l2": "flushed between launches" if small else "working set larger than L2"}), flush=True)
+        h.free()
+
+    which = args.suite.split(",")
+    if "cfg2" in which or "all" in which:
+        measure("config2", synth.config2(draw_input=False), 1)
+    if "resnet" in which or "all" in which:
+        for i in range(4):
+            for N in (1, 32):
+                measure("resnet50_fp16", synth.resnet50_layer(i, N=N, draw_input=False), N)
+    if "sweep" in which or "all" in which:
+        for npat in synth.SWEEP_PATTERNS:
+            for prune in synth.SWEEP_PRUNE:
+                L = synth.sweep_layer(npat, prune, N=64, draw_input=False)
+                measure("sweep", L, 64)
+                measure("sweep", L, 64, order=synth.random_filter_order(512, 7))
+                measure("sweep", L, 64, variant="tiled")
+                measure("sweep", L, 64, variant="tiled", order=synth.random_filter_order(512, 7))
+    if "ablation" in which or "all" in which:
+        seen = set()
+        for i in range(13):
+            if synth.VGG16_CONVS[i] in seen:
+                continue
+            seen.add(synth.VGG16_CONVS[i])
+            L = synth.vgg16_layer(i, N=1)
+            for variant in ("noopt", "reorder", "tiled", "dense_tc"):
+                measure("ablation_vgg_unique_layers", L, 1, variant=variant, reps=5 if variant in ("noopt", "reorder") else 20)
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -191,9 +273,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
+    ap.add_argument("--suite", default="", help="instead of the headline step: cfg2,resnet,sweep,ablation or all "
+                                                "(one JSON line per measured point)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.suite:
+        run_suite(args)
         return
     args.warmup = max(args.warmup, 3)
 

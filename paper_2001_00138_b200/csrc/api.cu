@@ -165,7 +165,9 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                     const double t_dense = terms * 2.0 * dp.taps * dp.Cp * dp.Fp * rows / 9.0e14 +
                                            static_cast<double>(desc->N) * desc->H * desc->W * (desc->C * 4.0 + dp.Cp * 2.0 * dp.S) / 4.0e12 +
                                            4e-6;
-                    const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / 1.2e13 + 4e-6;
+                    // CUDA-core kernel: ~12 TFLOP/s on kept weights for large images, ~4 for 14x14-class layers (measured)
+                    const double tiled_rate = (desc->H * desc->W <= 256) ? 4.0e12 : 1.2e13;
+                    const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / tiled_rate + 1.5e-5;
                     // layers with 9*C <= 64 (gathered-neighbourhood GEMM) are store-bound there: measured slower than the
                     // CUDA-core kernel on the RGB first layer, so AUTO leaves them on it unless it cannot run the layer
                     if (t_dense < t_tiled && (!dp.im2col || !can_tile)) h->variant = PATDNN_VARIANT_DENSE_TC;
