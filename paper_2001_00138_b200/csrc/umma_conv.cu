@@ -161,13 +161,16 @@ __global__ void __launch_bounds__(256) transition_kernel(T *__restrict__ src, ui
                     v = __half2float(sp[0]);
                     if (pool) v = fmaxf(fmaxf(v, __half2float(sp[1])), fmaxf(__half2float(sp[Ws]), __half2float(sp[Ws + 1])));
                 } else {
-                    if (pool) {
+                    if (pool && (Ws & 1) == 0 && (reinterpret_cast<uintptr_t>(src) & 7) == 0) {   // 8-byte aligned pairs
                         const float2 a = *reinterpret_cast<const float2 *>(sp), b = *reinterpret_cast<const float2 *>(sp + Ws);
                         v = fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y));
                         if (clear) {
                             *reinterpret_cast<float2 *>(sp) = make_float2(0.f, 0.f);
                             *reinterpret_cast<float2 *>(sp + Ws) = make_float2(0.f, 0.f);
                         }
+                    } else if (pool) {                       // odd row pitch: the pairs are not 8-byte aligned
+                        v = fmaxf(fmaxf(sp[0], sp[1]), fmaxf(sp[Ws], sp[Ws + 1]));
+                        if (clear) { sp[0] = 0.f; sp[1] = 0.f; sp[Ws] = 0.f; sp[Ws + 1] = 0.f; }
                     } else {
                         v = sp[0];
                         if (clear) sp[0] = 0.f;

@@ -153,6 +153,42 @@ def test_vgg_stack_reduced_spatial_per_layer_and_chained():
         h.free()
 
 
+@pytest.mark.parametrize("variants", [("dense", "dense", "dense"), ("tiled", "dense", "tiled"), ("dense", "tiled", "dense"),
+                                      ("reorder", "dense", "dense")])
+@pytest.mark.parametrize("hw", [(7, 7), (13, 9), (6, 10), (5, 3)])
+def test_small_stack_with_odd_sizes_and_pools(variants, hw):
+    """Three chained layers with a pool after the first two, on extents that are odd before and after pooling, with
+    every hand-over between the kernel families (NCHW <-> channels-innermost split operands, pooled or not)."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, (H, W) = 3, hw
+    chans = [5, 70, 24, 9]
+    x = synth.make_layer("x", F=1, C=chans[0], N=N, H=H, W=W, seed=5, x_dist="normal").x
+    cur, handles, h, w = x, [], H, W
+    for i in range(3):
+        L = synth.make_layer(f"s{i}", F=chans[i + 1], C=chans[i], N=N, H=h, W=w, seed=900 + i, prune=0.4, bias_std=0.3,
+                             draw_input=False)
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=h, W=w, relu=True, bias=L.bias,
+                                variant=VARIANTS[variants[i]]))
+        cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+        if i < 2 and h >= 2 and w >= 2:
+            cur = oracle.maxpool2x2(cur)
+            h, w = h // 2, w // 2
+    pools = [1 if (i < 2) else 0 for i in range(3)]
+    if cur.shape[2:] != (h, w) or H // 2 // 2 < 1 or W // 2 // 2 < 1:
+        pytest.skip("extent too small for two pools")
+    stack = B.Stack(handles, pools)
+    assert stack.out_shape() == cur.shape
+    out = torch.empty(cur.shape, device="cuda")
+    stack.run(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert_close(out.cpu().numpy(), cur, 4 * TOL_F32, f"stack {variants} {hw}")
+    stack.free()
+    for hd in handles:
+        hd.free()
+
+
 @pytest.mark.parametrize("i,N", [(0, 32), (1, 32), (5, 32), (12, 32), (3, 1), (8, 1), (11, 1)])
 def test_vgg_full_size_sampled(i, N):
     """Full-size layers in the benchmark's launch configuration; outputs sampled and checked one by one."""
