@@ -99,6 +99,8 @@ __global__ void __launch_bounds__(256) conv_noopt_kernel(SimpleParams p) {
 
 template <typename T>
 __global__ void __launch_bounds__(256) maxpool2x2_kernel(const T *in, T *out, int NC, int H, int W) {
+    pdl_trigger();
+    pdl_wait();
     const int Ho = H / 2, Wo = W / 2;
     const size_t total = static_cast<size_t>(NC) * Ho * Wo;
     for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
@@ -112,6 +114,11 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const T *in, T *out, in
         const float b = fmaxf(to_f32<T>(p[W]), to_f32<T>(p[W + 1]));
         out[idx] = from_f32<T>(fmaxf(a, b));
     }
+}
+
+bool pdl_enabled() {
+    static const bool on = [] { const char *v = std::getenv("PATDNN_PDL"); return !(v && v[0] == '0'); }();
+    return on;
 }
 
 cudaError_t launch_simple(const SimpleParams &p, int variant, int dtype, cudaStream_t stream) {
@@ -132,12 +139,11 @@ cudaError_t launch_maxpool2x2(const void *in, void *out, int N, int C, int H, in
     if (total == 0) return cudaSuccess;
     const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 16));
     if (dtype == 1)
-        maxpool2x2_kernel<__half><<<blocks, 256, 0, stream>>>(static_cast<const __half *>(in),
-                                                              static_cast<__half *>(out), N * C, H, W);
+        return launch_pdl(maxpool2x2_kernel<__half>, dim3(blocks), dim3(256), 0, stream, 1, static_cast<const __half *>(in),
+                          static_cast<__half *>(out), N * C, H, W);
     else
-        maxpool2x2_kernel<float><<<blocks, 256, 0, stream>>>(static_cast<const float *>(in),
-                                                             static_cast<float *>(out), N * C, H, W);
-    return cudaGetLastError();
+        return launch_pdl(maxpool2x2_kernel<float>, dim3(blocks), dim3(256), 0, stream, 1, static_cast<const float *>(in),
+                          static_cast<float *>(out), N * C, H, W);
 }
 
 }  // namespace patdnn

@@ -94,6 +94,8 @@ __global__ void __launch_bounds__(PW *FW * 32, MINB) conv_tiled_kernel(const Til
     constexpr int NT = PW * FW * 32;
     constexpr int ES = sizeof(T);
     extern __shared__ __align__(16) unsigned char smem[];
+    pdl_trigger();
+    pdl_wait();                                  // the input may be the previous kernel's output
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int fw = warp % FW, pw = warp / FW;
@@ -242,8 +244,7 @@ cudaError_t launch_instance(const TiledPlan &plan, const TiledParams &p, cudaStr
     if (prepare_only)   // per kernel instance, not per layer: the largest opt-in size
         return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
     const int grid = plan.grid_pix * plan.grid_fg;
-    kern<<<grid, PW * FW * 32, plan.smem_bytes, stream>>>(p);
-    return cudaGetLastError();
+    return launch_pdl(kern, dim3(grid), dim3(PW * FW * 32), plan.smem_bytes, stream, 1, p);
 }
 
 

@@ -77,7 +77,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *st
             "selp.b32 %0, 1, 0, P1;\n\t}"
             : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
-        if (*reinterpret_cast<volatile int *>(status) != 0) return false;      // another role already gave up
+        // another role already gave up?  (a global read: only now and then, it would otherwise sit on every wake-up path)
+        if ((i & 15u) == 15u && *reinterpret_cast<volatile int *>(status) != 0) return false;
     }
     atomicCAS(status, 0, code);
     return false;
@@ -144,6 +145,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) transition_kernel(T *__restrict__ src, uint16_t *__restrict__ dst,
                                                          const float *__restrict__ bias, int relu, int pool, int clear,
                                                          int N, int C, int Hs, int Ws, int Cp, int S) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float tile[64][33];
     const int H = pool ? Hs / 2 : Hs, W = pool ? Ws / 2 : Ws;
     const int cblocks = Cp / 64;
@@ -211,6 +214,8 @@ template <bool POOL>
 __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__ src, uint16_t *__restrict__ dst,
                                                              const float *__restrict__ bias, int relu, int clear,
                                                              int N, int C, int Hs, int Ws, int Cp, int S) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int XT = POOL ? 32 : 64;
     __shared__ float tile[64][XT + 1];
     const int H = POOL ? Hs / 2 : Hs, W = POOL ? Ws / 2 : Ws;
@@ -291,6 +296,8 @@ __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__
 template <typename T>
 __global__ void __launch_bounds__(256) im2col_kernel(const T *__restrict__ src, uint16_t *__restrict__ dst, int N, int C,
                                                       int H, int W, int S) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float rows[7][3][36];                             // [channel][row -1..1][column -1..32 (+pad)]
     const int x0 = blockIdx.x * 32, y = blockIdx.y, n = blockIdx.z;
     for (int i = threadIdx.x; i < C * 3 * 34; i += 256) {
@@ -413,6 +420,8 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) PATDNN_STAMP(0);
+    pdl_trigger();
     const int stages = p.stages;
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[8]), bar_acc = smem_u32(&bars[16]);
     int *status = p.status;
@@ -453,6 +462,8 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
+    if (threadIdx.x == 0) PATDNN_STAMP(1);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -480,6 +491,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 const int s = it % stages, use = it / stages;
                 ok = mbar_wait(bar_full + 8 * s, use & 1, status, 2);
                 if (!ok) break;
+                if (it == 0) PATDNN_STAMP(2);
                 tc_fence_after();
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
                 const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + A_BYTES);
@@ -501,10 +513,12 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 umma_commit(bar_empty + 8 * s);                 // frees the stage once these MMAs have read it
             }
             if (ok) umma_commit(bar_acc);
+            PATDNN_STAMP(3);
         }
     } else {
         // epilogue warps: warp w owns TMEM lanes 32*(w%4) .. +31; lane = output pixel m of the box
         if (mbar_wait(bar_acc, 0, status, 3)) {
+            if (threadIdx.x == 64) PATDNN_STAMP(4);
             tc_fence_after();
             if (ks == 1) {
 #pragma unroll 1
@@ -564,8 +578,10 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         }
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
+    if (threadIdx.x == 64) PATDNN_STAMP(5);
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) PATDNN_STAMP(6);
     if (warp == 2) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
@@ -610,6 +626,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     const int nshift = p.taps == 9 ? 3 : 1;                     // 3 horizontal shifts x 3 vertical taps, or one gathered tap
 
     if (threadIdx.x == 0) PATDNN_STAMP(0);
+    pdl_trigger();
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
             mbar_init(bar_fa + 8 * s, 1); mbar_init(bar_ea + 8 * s, 1);
@@ -627,6 +644,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
     if (threadIdx.x == 0) PATDNN_STAMP(1);
 
     auto decode = [&](int t, int &ft, int &x0, int &y0, int &n) {
@@ -798,25 +816,14 @@ template <int BN, int TERMS, typename T>
 cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_kernel<BN, TERMS, T>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-    if (pl.ksplit == 1) {
-        kern<<<pl.grid, kThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
-        return cudaGetLastError();
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pl.grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = pl.smem_bytes; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = pl.ksplit; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, pl.mapA, pl.mapB, p);
+    return launch_pdl(kern, dim3(pl.grid), dim3(kThreads), pl.smem_bytes, st, pl.ksplit, pl.mapA, pl.mapB, p);
 }
 
 template <int BN, int MT, int TERMS, typename T>
 cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-    kern<<<pl.grid, kHaloThreads, pl.smem_bytes, st>>>(pl.mapA, pl.mapB, p);
-    return cudaGetLastError();
+    return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, p);
 }
 
 cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
@@ -1027,32 +1034,29 @@ cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const
     const int gz = N * (Cp / 64);
     if (!src_is_half && Ws % 4 == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
         float *fs = static_cast<float *>(const_cast<void *>(src));
+        uint16_t *d16 = static_cast<uint16_t *>(dst);
         if (pool)
-            transition_vec_kernel<true><<<dim3((W + 31) / 32, H, gz), 256, 0, st>>>(fs, static_cast<uint16_t *>(dst), bias, relu,
-                                                                                     clear, N, C, Hs, Ws, Cp, S);
-        else
-            transition_vec_kernel<false><<<dim3((W + 63) / 64, H, gz), 256, 0, st>>>(fs, static_cast<uint16_t *>(dst), bias, relu,
-                                                                                      clear, N, C, Hs, Ws, Cp, S);
-        return cudaGetLastError();
+            return launch_pdl(transition_vec_kernel<true>, dim3((W + 31) / 32, H, gz), dim3(256), 0, st, 1, fs, d16, bias, relu, clear,
+                              N, C, Hs, Ws, Cp, S);
+        return launch_pdl(transition_vec_kernel<false>, dim3((W + 63) / 64, H, gz), dim3(256), 0, st, 1, fs, d16, bias, relu, clear,
+                          N, C, Hs, Ws, Cp, S);
     }
     dim3 grid((W + 31) / 32, H, gz), block(32, 8);
     if (src_is_half)
-        transition_kernel<__half><<<grid, block, 0, st>>>(static_cast<__half *>(const_cast<void *>(src)),
-                                                          static_cast<uint16_t *>(dst), bias, relu, pool, 0, N, C, Hs, Ws, Cp, S);
-    else
-        transition_kernel<float><<<grid, block, 0, st>>>(static_cast<float *>(const_cast<void *>(src)),
-                                                         static_cast<uint16_t *>(dst), bias, relu, pool, clear, N, C, Hs, Ws, Cp, S);
-    return cudaGetLastError();
+        return launch_pdl(transition_kernel<__half>, grid, block, 0, st, 1, static_cast<__half *>(const_cast<void *>(src)),
+                          static_cast<uint16_t *>(dst), bias, relu, pool, 0, N, C, Hs, Ws, Cp, S);
+    return launch_pdl(transition_kernel<float>, grid, block, 0, st, 1, static_cast<float *>(const_cast<void *>(src)),
+                      static_cast<uint16_t *>(dst), bias, relu, pool, clear, N, C, Hs, Ws, Cp, S);
 }
 
 cudaError_t launch_im2col(const void *src, int src_is_half, void *dst, int N, int C, int H, int W, int S, cudaStream_t st) {
     if (N == 0) return cudaSuccess;
     dim3 grid((W + 31) / 32, H, N);
     if (src_is_half)
-        im2col_kernel<__half><<<grid, 256, 0, st>>>(static_cast<const __half *>(src), static_cast<uint16_t *>(dst), N, C, H, W, S);
-    else
-        im2col_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float *>(src), static_cast<uint16_t *>(dst), N, C, H, W, S);
-    return cudaGetLastError();
+        return launch_pdl(im2col_kernel<__half>, grid, dim3(256), 0, st, 1, static_cast<const __half *>(src),
+                          static_cast<uint16_t *>(dst), N, C, H, W, S);
+    return launch_pdl(im2col_kernel<float>, grid, dim3(256), 0, st, 1, static_cast<const float *>(src), static_cast<uint16_t *>(dst),
+                      N, C, H, W, S);
 }
 
 cudaError_t launch_dense_gemm(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st) {
