@@ -399,7 +399,7 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->entries = p.entries;
     } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         const DensePlan &p = h->dense;
-        info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 6;
+        info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 10;
         info->channels_per_stage = 64; info->channel_splits = p.ksplit;
         info->grid_x = p.grid; info->grid_y = p.halo ? p.n_tiles : 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
         info->entries = static_cast<int64_t>(p.taps) * p.Fp * p.Cp;

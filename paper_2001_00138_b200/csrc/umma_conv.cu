@@ -24,6 +24,7 @@
 // Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves through the normal exit
 // (TMEM is always deallocated).  No cluster multicast anywhere.
 #include <cuda.h>
+#include <type_traits>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -39,12 +40,12 @@
 namespace patdnn {
 
 #ifdef PATDNN_TRACE
-// Debug-only CTA timeline (build with -DPATDNN_TRACE): 8 time stamps per CTA, read back by patdnn_trace_read().
+// Debug-only CTA timeline (build with -DPATDNN_TRACE): up to 16 time stamps per CTA, read back by patdnn_trace_read().
 __device__ unsigned long long g_trace[1 << 16];
 __device__ __forceinline__ void trace_stamp(int slot) {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (blockIdx.x < (1 << 13)) g_trace[blockIdx.x * 8 + slot] = t;
+    if (blockIdx.x < (1 << 12)) g_trace[blockIdx.x * 16 + slot] = t;
 }
 #define PATDNN_STAMP(slot) trace_stamp(slot)
 #else
@@ -53,7 +54,7 @@ __device__ __forceinline__ void trace_stamp(int slot) {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                // general kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kTileM = 128;
 constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
@@ -439,8 +440,11 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int total_iters = p.taps * p.KB;                      // taps = 9, or 1 for gathered (im2col) activations
     const int it0 = rank * total_iters / ks;                    // even split: every range holds at least one iteration
     const int iters = (rank + 1) * total_iters / ks - it0;
-    // output pixel of this thread when it acts as an epilogue thread (warps 2..5 cover the 128 accumulator rows)
+    // output pixel of this thread when it acts as an epilogue thread (warps 2..5 and 6..9 each cover the 128 accumulator rows)
     const int q = warp & 3;
+    const int half = (warp - 2) >> 2;                           // epilogue warps 2..5 take the lower columns, 6..9 the upper
+    constexpr int HC = BN >= 64 ? BN / 2 : BN;                  // columns per half (narrow tiles: half 0 takes them all)
+    const int col_lo = (BN >= 64) ? half * HC : 0, col_hi = (BN >= 64) ? col_lo + HC : (half == 0 ? BN : 0);
     const int m = q * 32 + lane;
     const int per_img = p.TW * p.TH;
     const int tn = m / per_img, rem = m - tn * per_img;
@@ -464,6 +468,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t tmem_base = tmem_slot;
     pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
     if (threadIdx.x == 0) PATDNN_STAMP(1);
+    bool acc_ready = false;                                     // epilogue thread holding a finished K-range partial
 
     if (warp == 0) {
         if (lane == 0) {
@@ -522,7 +527,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             tc_fence_after();
             if (ks == 1) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = col_lo; c0 < col_hi; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
                     float a[32];
@@ -536,49 +541,63 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     emit_chunk<32, T>(p, a, s_bias + c0, f0 + c0, n, y, x, pix_ok);
                 }
             } else {
-                // partial sums of this K range -> own shared memory, column-major [BN][128] (pipeline buffers are free)
-                float *R = reinterpret_cast<float *>(smem);
-#pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    uint32_t v[32], v2[32];
-                    tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
-                    if constexpr (MERGE) tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + BN + c0, v2);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        R[(c0 + j) * kTileM + m] = __uint_as_float(v[j]) + (MERGE ? __uint_as_float(v2[j]) : 0.f);
-                }
+                acc_ready = true;                                // partial sums stay in TMEM until the cluster is ready
             }
         }
     }
     if (ks > 1) {
-        // Sum the K ranges across the cluster through distributed shared memory: CTA r finishes columns
-        // [r*BN/ks, (r+1)*BN/ks).  Every thread of every CTA takes part in both cluster barriers, also after a
-        // timed-out wait, so nobody is left waiting.
+        // Sum the K ranges across the cluster through distributed shared memory.  CTA r finishes the columns
+        // [r*BN/ks, (r+1)*BN/ks): every CTA PUSHES the matching slice of its partial tile into r's shared memory
+        // (remote stores need no answer, remote loads would expose their latency; a warp stores 128 contiguous bytes --
+        // 16-byte stores scattered at a row pitch measured twice as slow), slot = sender's rank, layout
+        // [slot][column][pixel]; then r adds
+        // the ks slots in rank order from its own memory.  Barrier 1: every CTA's MMAs have read their pipeline
+        // buffers, which the slots reuse.  Barrier 2: all slots have landed.  Every thread of every CTA takes part in
+        // both barriers, also after a timed-out wait, so nobody is left waiting.
+        const int cols = BN / ks;
+        const uint32_t rbase = smem_u32(smem);
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (warp >= 2) {
-            const int cols = BN / ks, cbeg = rank * cols;
-            const uint32_t rbase = smem_u32(smem);
+        if (threadIdx.x == 64) PATDNN_STAMP(7);
+        if (acc_ready) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < cols; c0 += 8) {
+            for (int c0 = col_lo; c0 < col_hi; c0 += 32) {
+                uint32_t v[32], v2[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0, v);
+                if constexpr (MERGE) tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + BN + c0, v2);
+#pragma unroll
+                for (int j0 = 0; j0 < 32; j0 += 8) {             // cols is a multiple of 8: one owner per 8 columns
+                    const int owner = (c0 + j0) / cols, cl = (c0 + j0) - owner * cols;
+                    uint32_t remote;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(rbase), "r"(owner));
+                    remote += ((rank * cols + cl) * kTileM + m) * 4;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float val = __uint_as_float(v[j0 + j]) + (MERGE ? __uint_as_float(v2[j0 + j]) : 0.f);
+                        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote + j * kTileM * 4), "f"(val) : "memory");
+                    }
+                }
+            }
+        }
+        if (threadIdx.x == 64) PATDNN_STAMP(8);
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (threadIdx.x == 64) PATDNN_STAMP(9);
+        if (warp >= 2) {
+            const float *R = reinterpret_cast<const float *>(smem);
+            const int cbeg = rank * cols;
+#pragma unroll 1
+            for (int c0 = 8 * half; c0 < cols; c0 += 16) {
                 float a[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) a[j] = 0.f;
-                for (int qq = 0; qq < ks; ++qq) {
-                    uint32_t remote;
-                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(rbase), "r"(qq));
+                for (int qq = 0; qq < ks; ++qq)
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float t;
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(t) : "r"(remote + ((cbeg + c0 + j) * kTileM + m) * 4) : "memory");
-                        a[j] += t;
-                    }
-                }
+                    for (int j = 0; j < 8; ++j) a[j] += R[(qq * cols + c0 + j) * kTileM + m];
                 emit_chunk<8, T>(p, a, s_bias + cbeg + c0, f0 + cbeg + c0, n, y, x, pix_ok);
             }
         }
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (threadIdx.x == 64) PATDNN_STAMP(5);
     }
-    if (threadIdx.x == 64) PATDNN_STAMP(5);
+    if (ks == 1 && threadIdx.x == 64) PATDNN_STAMP(5);
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) PATDNN_STAMP(6);
@@ -879,13 +898,17 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     // scheduling cost more than the shorter loop saves); if that still leaves most SMs idle, narrow the filter tile.
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
     const int total_iters = pl.taps * pl.KB;
+    // a 2-way split of a 128-wide tile exchanges a quarter of what a 4-way split of a 256-wide tile does (measured faster)
+    while (pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 < 100) pl.BN /= 2;
     while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 4 < 100) pl.BN /= 2;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
     int ks = 1;
+    // one wave only: with ~200 KB of shared memory per CTA, 148 CTAs fit as clusters of 2, 132 as clusters of 4
+    // (occupancy query); a second wave costs more than the shorter loop saves
     if (base_grid < 100)
-        while (ks < 4 && base_grid * ks * 2 <= 296 && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
+        while (ks < 4 && base_grid * ks * 2 <= (ks * 2 == 2 ? 148 : 132) && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
     if (const char *ov = std::getenv("PATDNN_KSPLIT")) {
         const int want = atoi(ov);
         if ((want == 1 || want == 2 || want == 4 || want == 8) && want <= total_iters && pl.BN / want >= 8) ks = want;
