@@ -71,6 +71,8 @@ struct patdnn_layer {
     int *d_status = nullptr;
     DensePlan dense_static;                  // same plan with its activation map over the fixed scratch array
     bool dense_static_ready = false;
+    DensePlan dense_pool;                    // plan over the same buffers whose epilogue can max-pool (built by a stack)
+    int dense_pool_state = 0;                // 0 = not tried, 1 = ready, -1 = this layer's shape has no such plan
     // staging buffers of patdnn_conv_host
     void *d_in_stage = nullptr, *d_out_stage = nullptr;
 };
@@ -99,11 +101,13 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
 
 // GEMM of a tensor-core layer whose split activations already sit in the buffer its activation map points to.
 // next == nullptr: finished NCHW result into `out`; else the result goes, already split and channels-innermost, straight
-// into the activation buffer of the tensor-core layer `next` (same spatial size, no pooling in between).
-static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const patdnn_layer *next, cudaStream_t st) {
+// into the activation buffer of the tensor-core layer `next` (same spatial size; or, with `pooled` and a poolable
+// plan, after a 2x2 max-pool taken in the epilogue).
+static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const patdnn_layer *next, cudaStream_t st,
+                      bool pooled = false) {
     DenseParams p = dense_params(h, pl);
     if (next) {
-        p.mode = 3; p.out = next->d_act; p.out_cp = next->dense.Cp;
+        p.mode = pooled ? 4 : 3; p.out = next->d_act; p.out_cp = next->dense.Cp;
     } else {
         p.mode = 0; p.out = out;
     }
@@ -447,6 +451,23 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         s->layers.push_back(h);
         s->pool.push_back(pool);
     }
+    // tensor-core layer -> pool -> tensor-core layer: a second plan of the first layer whose epilogue pools in registers
+    for (int i = 0; i + 1 < n; ++i) {
+        patdnn_layer *h = s->layers[i], *nx = s->layers[i + 1];
+        if (!s->pool[i] || h->variant != PATDNN_VARIANT_DENSE_TC || nx->variant != PATDNN_VARIANT_DENSE_TC || nx->dense.im2col ||
+            h->dense_pool_state != 0)
+            continue;
+        const patdnn_desc &d = h->desc;
+        h->dense_pool_state = -1;
+        if (d.N < 1) continue;
+        DensePlan pp;
+        plan_dense(d.F, d.C, d.N, d.H, d.W, d.dtype, pp, true, h->dense.BN);
+        if (!pp.poolable || pp.Fp != h->dense.Fp || pp.Cp != h->dense.Cp || pp.taps != h->dense.taps) continue;
+        if (make_dense_maps(pp, h->d_act, h->d_wdense, d.N, d.H, d.W, d.dtype) != PATDNN_OK) continue;
+        if (prepare_dense(pp, d.dtype) != cudaSuccess) { cudaGetLastError(); continue; }
+        h->dense_pool = pp;
+        h->dense_pool_state = 1;
+    }
     s->oN = N; s->oF = C; s->oH = H; s->oW = W;
     s->buf_bytes = std::max<size_t>(max_bytes, 16);
     const patdnn_desc &d0 = handles[0]->desc;
@@ -462,7 +483,8 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
 
 // Chained execution.  Where two tensor-core layers follow each other without a pool, the first one's epilogue writes
 // the second one's input directly (bias + ReLU applied, channels innermost, operands split): no tensor in NCHW form and
-// no layout kernel in between.  A pool between them is folded into the layout kernel of the second.
+// no layout kernel in between.  A pool between them is taken in the first one's epilogue where its shape allows a
+// poolable plan, else folded into the layout kernel of the second.
 int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
     if (!s || !in || !out) return PATDNN_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -495,15 +517,15 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
                 if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
-            patdnn_layer *next = (!last && !s->pool[i] && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC &&
-                                  !s->layers[i + 1]->dense.im2col)
-                                     ? s->layers[i + 1] : nullptr;
+            const bool next_dense = !last && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC && !s->layers[i + 1]->dense.im2col;
+            const bool fuse_pool = next_dense && s->pool[i] && h->dense_pool_state == 1;
+            patdnn_layer *next = (next_dense && (!s->pool[i] || fuse_pool)) ? s->layers[i + 1] : nullptr;
             void *dst = next ? nullptr : ((last && !s->pool[i]) ? out : s->buf[which]);
-            const int rc = dense_gemm(h, h->dense, dst, next, st);
+            const int rc = dense_gemm(h, fuse_pool ? h->dense_pool : h->dense, dst, next, st, fuse_pool);
             if (rc) return rc;
             direct = next != nullptr;
             if (!direct) { cur = dst; which ^= 1; }
-            cur_pool = s->pool[i] != 0;
+            cur_pool = s->pool[i] != 0 && !fuse_pool;
             curH = d.H; curW = d.W;
         } else {
             if (cur_pool) {

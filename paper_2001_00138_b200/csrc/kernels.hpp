@@ -135,6 +135,7 @@ struct DensePlan {
     int n_tiles = 0;                       // halo kernel: tiles shared by the persistent CTAs
     int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
+    int poolable = 0;                      // boxes meet the conditions of the fused max-pool epilogue (mode 4)
     CUtensorMap mapA{}, mapB{};
 };
 
@@ -146,15 +147,19 @@ struct DenseParams {
     int TW, TH, TN, tiles_x, tiles_y, n_ftiles;
     int KB, stages, box_bytes, relu;
     int tiles_n, iters_per_split, ksplit, na, taps;
-    int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer
-    int out_cp;                 // channel pitch of the mode-3 destination
+    int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer;
+                                // 4: as 3 after a fused 2x2 max-pool, [S][N][H/2][W/2][out_cp] (needs a pool_tiles plan)
+    int out_cp;                 // channel pitch of the mode-3/4 destination
 };
 
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static
 int static_scratch_address(void **ptr);                    // PATDNN_* status; first call per device looks the address up
 
 bool dense_supported(int F, int C, int N, int H, int W);
-void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl);
+// pool_tiles: only pixel boxes whose epilogue can max-pool in registers (one image per box, 2/4/8/16 pixels wide, starting
+// on even rows); sets pl.poolable.  force_bn pins the filter tile width, so that a second plan of a layer shares the
+// weight layout of the first.
+void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, bool pool_tiles = false, int force_bn = 0);
 void build_dense_weights(const Fkw &fkw, const DensePlan &pl, std::vector<uint16_t> &w);
 int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, int dtype);
 cudaError_t prepare_dense(const DensePlan &pl, int dtype);

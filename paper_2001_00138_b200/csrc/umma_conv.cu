@@ -344,10 +344,11 @@ __global__ void __launch_bounds__(256) im2col_kernel(const T *__restrict__ src, 
 }
 
 // Finish CNT consecutive filters (f_lo ..) of one output pixel: bias + ReLU, then either the caller's NCHW tensor
-// (mode 0) or the next tensor-core layer's split channels-innermost activations (mode 3: [S][N][H][W][out_cp]).
+// (mode 0) or the next tensor-core layer's split channels-innermost activations (mode 3: [S][N][H][W][out_cp];
+// mode 4: the same after a fused 2x2 max-pool, [S][N][H/2][W/2][out_cp]).
 template <int CNT, typename T>
 __device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT], const float *s_bias, int f_lo, int n, int y,
-                                           int x, bool pix_ok) {
+                                           int x, bool pix_ok) {   // called by whole warps (mode 4 exchanges between lanes)
     // s_bias: this CTA's bias slice in shared memory, indexed from f_lo (zero beyond the layer's last filter)
 #pragma unroll
     for (int j = 0; j < CNT; ++j) {
@@ -355,6 +356,20 @@ __device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT]
         float v = a[j] + s_bias[j];
         if (p.relu) v = fmaxf(v, 0.f);
         a[j] = (f < p.F) ? v : 0.f;
+    }
+    if (p.mode == 4) {
+        // Fused 2x2/stride-2 max-pool (bias and ReLU commute with the maximum): the four pixels of a window sit in one
+        // warp -- x and x+1 in neighbouring lanes, y and y+1 TW lanes apart (TW is 2, 4, 8 or 16 and boxes start on even
+        // coordinates in this mode) -- so two butterfly exchanges leave the window maximum in all four lanes, and the
+        // lane of the even/even pixel stores it at the pooled position.
+#pragma unroll
+        for (int j = 0; j < CNT; ++j) {
+            float v = a[j];
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, p.TW));
+            a[j] = v;
+        }
+        pix_ok = pix_ok && !(x & 1) && !(y & 1) && x + 1 < p.W && y + 1 < p.H;
     }
     if (!pix_ok) return;
 #ifdef PATDNN_TRACE
@@ -375,8 +390,10 @@ __device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT]
     } else {
         if (f_lo >= p.out_cp) return;                    // filter tiles may be padded beyond the next layer's channels
         uint16_t *dst = static_cast<uint16_t *>(p.out);
-        const size_t o = ((static_cast<size_t>(n) * p.H + y) * p.W + x) * p.out_cp + f_lo;
-        const size_t plane_out = static_cast<size_t>(p.N) * p.H * p.W * p.out_cp;
+        const int oh = p.mode == 4 ? p.H / 2 : p.H, ow = p.mode == 4 ? p.W / 2 : p.W;
+        const int oy = p.mode == 4 ? y >> 1 : y, ox = p.mode == 4 ? x >> 1 : x;
+        const size_t o = ((static_cast<size_t>(n) * oh + oy) * ow + ox) * p.out_cp + f_lo;
+        const size_t plane_out = static_cast<size_t>(p.N) * oh * ow * p.out_cp;
 #pragma unroll
         for (int g = 0; g < CNT / 8; ++g) {
             uint32_t hi[4], lo[4];
@@ -869,7 +886,7 @@ bool dense_supported(int F, int C, int N, int H, int W) {
 }
 
 // Pixel box (TW x TH x TN <= 128) that wastes the fewest MMA rows for this image size.
-void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
+void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, bool pool_tiles, int force_bn) {
     pl = DensePlan();
     pl.S = dtype == PATDNN_F16 ? 1 : 2;
     pl.im2col = (9 * C <= kKBlock) ? 1 : 0;                        // tiny C: taps gathered into the channel dimension
@@ -886,8 +903,12 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     double best = -1;
     for (int tw = 1; tw <= std::min(W, kTileM); ++tw) {
         const int th = std::min(H, kTileM / tw);
-        const int tn = (th == H) ? std::max(1, std::min(N, kTileM / (tw * th))) : 1;
+        int tn = (th == H) ? std::max(1, std::min(N, kTileM / (tw * th))) : 1;
         if (tw > 256 || th > 256 || tn > 256) continue;
+        if (pool_tiles) {                                           // see emit_chunk, mode 4
+            if (!(tw == 2 || tw == 4 || tw == 8 || tw == 16) || ((th & 1) && th != H)) continue;
+            tn = 1;
+        }
         const int64_t tx = (W + tw - 1) / tw, ty = (H + th - 1) / th, tz = (N + tn - 1) / tn;
         const double util = static_cast<double>(N) * H * W / (static_cast<double>(tx * ty * tz) * kTileM);
         const double score = util + 1e-6 * tw;                      // prefer wide boxes (coalesced stores) on ties
@@ -901,6 +922,8 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
     // a 2-way split of a 128-wide tile exchanges a quarter of what a 4-way split of a 256-wide tile does (measured faster)
     while (pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 < 100) pl.BN /= 2;
     while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 4 < 100) pl.BN /= 2;
+    if (force_bn) pl.BN = force_bn;
+    pl.poolable = (pool_tiles && best > 0) ? 1 : 0;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
@@ -928,6 +951,7 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl) {
         const double util_now = static_cast<double>(N) * H * W / (static_cast<double>(ptiles) * kTileM);
         int btw = 0; double butil = 0;
         for (int tw : {32, 16, 8, 64, 128}) {                      // ties: 32-wide boxes first (128-byte store rows, 1.5x halo)
+            if (pool_tiles && tw != 16 && tw != 8) continue;
             const int th = kTileM / tw;
             const double u = static_cast<double>(H) * W /
                              (static_cast<double>((W + tw - 1) / tw) * tw * static_cast<double>((H + th - 1) / th) * th);

@@ -181,8 +181,12 @@ def test_small_stack_with_odd_sizes_and_pools(variants, hw):
     stack = B.Stack(handles, pools)
     assert stack.out_shape() == cur.shape
     out = torch.empty(cur.shape, device="cuda")
+    B.reset_launch_count()
     stack.run(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
+    if variants == ("dense", "dense", "dense"):
+        # one layout kernel for the caller's NCHW input, then three GEMMs: both pools are taken in the epilogues
+        assert B.launch_count() == 4
     assert_close(out.cpu().numpy(), cur, 4 * TOL_F32, f"stack {variants} {hw}")
     stack.free()
     for hd in handles:
