@@ -104,8 +104,9 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
 // into the activation buffer of the tensor-core layer `next` (same spatial size; or, with `pooled` and a poolable
 // plan, after a 2x2 max-pool taken in the epilogue).
 static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const patdnn_layer *next, cudaStream_t st,
-                      bool pooled = false) {
+                      bool pooled = false, const void *gather_src = nullptr) {
     DenseParams p = dense_params(h, pl);
+    p.gather_src = gather_src;                               // gather plans read the layer's NCHW input themselves
     if (next) {
         p.mode = pooled ? 4 : 3; p.out = next->d_act; p.out_cp = next->dense.Cp;
     } else {
@@ -123,6 +124,7 @@ static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const pat
 // One tensor-core layer from an NCHW input to its finished NCHW output.
 static int dense_forward(patdnn_layer *h, const DensePlan &pl, const void *in, void *act, void *out, cudaStream_t st) {
     const patdnn_desc &d = h->desc;
+    if (pl.gather) return dense_gemm(h, pl, out, nullptr, st, false, in);
     cudaError_t e = pl.im2col ? launch_im2col(in, d.dtype == PATDNN_F16, act, d.N, d.C, d.H, d.W, pl.S, st)
                               : launch_transition(in, d.dtype == PATDNN_F16, act, nullptr, 0, 0, 0, d.N, d.C, d.H, d.W, pl.Cp, pl.S, st);
     if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
@@ -202,7 +204,9 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                         h->device_bytes = static_cast<int64_t>(wd.size()) * 2;
                     }
                     if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
-                    if (!rc) {
+                    if (!rc && h->dense.gather) {
+                        h->d_act = h->d_wdense;                  // never read: the tensor map only needs a valid base
+                    } else if (!rc) {
                         const size_t act_bytes = static_cast<size_t>(h->dense.S) * std::max(desc->N, 1) * desc->H *
                                                  desc->W * h->dense.Cp * 2;
                         cudaError_t ce = cudaMalloc(&h->d_act, act_bytes);
@@ -308,6 +312,7 @@ int patdnn_conv_static(patdnn_handle h, const void *in, void *out, void *stream)
     if (h->variant != PATDNN_VARIANT_DENSE_TC) return patdnn_conv(h, in, out, stream);   // no scratch on those paths
     const patdnn_desc &d = h->desc;
     if (d.N == 0) return PATDNN_OK;
+    if (h->dense.gather) return dense_forward(h, h->dense, in, nullptr, out, static_cast<cudaStream_t>(stream));   // no scratch
     const size_t need = static_cast<size_t>(h->dense.S) * d.N * d.H * d.W * h->dense.Cp * 2;
     if (need > kStaticScratchBytes) return PATDNN_E_SCRATCH;
     void *scratch = nullptr;
@@ -462,7 +467,7 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         if (d.N < 1) continue;
         DensePlan pp;
         plan_dense(d.F, d.C, d.N, d.H, d.W, d.dtype, pp, true, h->dense.BN);
-        if (!pp.poolable || pp.Fp != h->dense.Fp || pp.Cp != h->dense.Cp || pp.taps != h->dense.taps) continue;
+        if (!pp.poolable || pp.Fp != h->dense.Fp || pp.Cp != h->dense.Cp || pp.taps != h->dense.taps || (h->dense.gather && !pp.gather)) continue;   // a gather layer owns no activation buffer
         if (make_dense_maps(pp, h->d_act, h->d_wdense, d.N, d.H, d.W, d.dtype) != PATDNN_OK) continue;
         if (prepare_dense(pp, d.dtype) != cudaSuccess) { cudaGetLastError(); continue; }
         h->dense_pool = pp;
@@ -501,6 +506,9 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
         const bool last = (i == n - 1);
         const bool is_dense = h->variant == PATDNN_VARIANT_DENSE_TC;
         if (is_dense) {
+            const bool next_dense = !last && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC && !s->layers[i + 1]->dense.im2col;
+            const bool fuse_pool = next_dense && s->pool[i] && h->dense_pool_state == 1;
+            const DensePlan &use = fuse_pool ? h->dense_pool : h->dense;
             if (!direct && h->dense.im2col) {
                 if (cur_pool) {
                     const int rc = patdnn_maxpool2x2(cur, s->buf[which], d.N, d.C, curH, curW, d.dtype, stream);
@@ -508,20 +516,20 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
                     cur = s->buf[which];
                     which ^= 1;
                 }
-                cudaError_t e = launch_im2col(cur, d.dtype == PATDNN_F16, h->d_act, d.N, d.C, d.H, d.W, h->dense.S, st);
-                if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
-                g_launches.fetch_add(1, std::memory_order_relaxed);
+                if (!use.gather) {
+                    cudaError_t e = launch_im2col(cur, d.dtype == PATDNN_F16, h->d_act, d.N, d.C, d.H, d.W, h->dense.S, st);
+                    if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
+                    g_launches.fetch_add(1, std::memory_order_relaxed);
+                }
             } else if (!direct) {
                 cudaError_t e = launch_transition(cur, d.dtype == PATDNN_F16, h->d_act, nullptr, 0, cur_pool, 0, d.N, d.C,
                                                   curH, curW, h->dense.Cp, h->dense.S, st);
                 if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
-            const bool next_dense = !last && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC && !s->layers[i + 1]->dense.im2col;
-            const bool fuse_pool = next_dense && s->pool[i] && h->dense_pool_state == 1;
             patdnn_layer *next = (next_dense && (!s->pool[i] || fuse_pool)) ? s->layers[i + 1] : nullptr;
             void *dst = next ? nullptr : ((last && !s->pool[i]) ? out : s->buf[which]);
-            const int rc = dense_gemm(h, fuse_pool ? h->dense_pool : h->dense, dst, next, st, fuse_pool);
+            const int rc = dense_gemm(h, use, dst, next, st, fuse_pool, (use.gather && !direct) ? cur : nullptr);
             if (rc) return rc;
             direct = next != nullptr;
             if (!direct) { cur = dst; which ^= 1; }

@@ -135,6 +135,7 @@ struct DensePlan {
     int n_tiles = 0;                       // halo kernel: tiles shared by the persistent CTAs
     int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
+    int gather = 0;                        // im2col layer on the persistent kernel: operand rows gathered in the kernel
     int poolable = 0;                      // boxes meet the conditions of the fused max-pool epilogue (mode 4)
     CUtensorMap mapA{}, mapB{};
 };
@@ -150,6 +151,7 @@ struct DenseParams {
     int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer;
                                 // 4: as 3 after a fused 2x2 max-pool, [S][N][H/2][W/2][out_cp] (needs a pool_tiles plan)
     int out_cp;                 // channel pitch of the mode-3/4 destination
+    const void *gather_src;     // gather plans: the layer's NCHW input (fp32 or fp16 as the layer's dtype)
 };
 
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static

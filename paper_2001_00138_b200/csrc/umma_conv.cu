@@ -56,6 +56,7 @@ namespace {
 
 constexpr int kThreads = 320;                // general kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA warp, eight epilogue warps
+constexpr int kGatherThreads = 128;          // plus four gather warps for layers whose operand rows are built in the kernel
 constexpr int kTileM = 128;
 constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
 constexpr uint32_t kSpinLimit = 1u << 21;    // bounded mbarrier polling: each poll may block up to ~1 us (hint below)
@@ -631,8 +632,12 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // CTAs are persistent (one per SM, tiles taken round-robin) and the accumulator is double buffered in TMEM: while the
 // epilogue warps drain tile i, the MMA thread already works on tile i+1.
 // Rings: A (per channel block and shift), B (per channel block and tap), accumulator full/empty (2 buffers).
-template <int BN, int MT, int TERMS, typename T>
-__global__ void __launch_bounds__(kHaloThreads, 1)
+//
+// GATHER (layers with 9*C <= 64, one gathered tap): no activation tensor in memory at all.  Four extra warps read the
+// 3x3 neighbourhood of their pixels straight from the caller's NCHW input, split it, and write the [pixel][k] operand
+// rows (k = 9*c + tap, zero beyond 9*C) into the A ring in the swizzled layout a TMA load would have produced.
+template <int BN, int MT, int TERMS, typename T, bool GATHER>
+__global__ void __launch_bounds__(GATHER ? kHaloThreads + kGatherThreads : kHaloThreads, 1)
 conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
     constexpr int S = (TERMS == 3) ? 2 : 1;
     constexpr int B_BYTES = BN * 128;
@@ -665,7 +670,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     pdl_trigger();
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
-            mbar_init(bar_fa + 8 * s, 1); mbar_init(bar_ea + 8 * s, 1);
+            mbar_init(bar_fa + 8 * s, GATHER ? kGatherThreads / 32 : 1); mbar_init(bar_ea + 8 * s, 1);
             mbar_init(bar_fb + 8 * s, 1); mbar_init(bar_eb + 8 * s, 1);
         }
         mbar_init(bar_af, 1); mbar_init(bar_af + 8, 1);
@@ -700,14 +705,16 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 const int f0 = ft * BN;
                 for (int cb = 0; cb < KB && ok; ++cb) {
                     for (int sx = 0; sx < nshift && ok; ++sx) {
-                        const int sa = ia % NA, ua = ia / NA;
-                        if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
-                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
-                        mbar_expect_tx(bar_fa + 8 * sa, S * a_plane);
+                        if constexpr (!GATHER) {
+                            const int sa = ia % NA, ua = ia / NA;
+                            if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
+                            const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                            mbar_expect_tx(bar_fa + 8 * sa, S * a_plane);
 #pragma unroll
-                        for (int sp = 0; sp < S; ++sp)
-                            tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - (nshift >> 1), y0 - (nshift >> 1), n, sp);
-                        ++ia;
+                            for (int sp = 0; sp < S; ++sp)
+                                tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - (nshift >> 1), y0 - (nshift >> 1), n, sp);
+                            ++ia;
+                        }
                         for (int r = 0; r < nshift; ++r) {
                             const int sb = ib % NB, ub = ib / NB;
                             if (ub > 0 && !mbar_wait(bar_eb + 8 * sb, (ub - 1) & 1, status, 1)) { ok = false; break; }
@@ -778,6 +785,66 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 if (ok) umma_commit(bar_af + 8 * buf);
             }
             PATDNN_STAMP(3);
+        }
+    } else if (GATHER && warp >= kHaloThreads / 32) {
+        // gather warps: per tile (one A stage: KB = 1) they stage the input patch with its one-pixel border in shared
+        // memory (coalesced reads, zeros outside the image), then thread g builds the operand rows g, g+128, ...
+        const T *src = static_cast<const T *>(p.gather_src);
+        const int g = threadIdx.x - kHaloThreads;
+        const int ph = MT * p.TH + 2, pw = p.TW + 2, pplane = ph * pw;
+        float *patch = reinterpret_cast<float *>(smem_b + NB * b_stage);     // [C][ph][pw], behind the two rings
+        int ia = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++ia) {
+            int ft, x0, y0, n;
+            decode(t, ft, x0, y0, n);
+            for (int i = g; i < p.C * pplane; i += kGatherThreads) {
+                const int c = i / pplane, rem = i - c * pplane, py = rem / pw, px = rem - py * pw;
+                const int yy = y0 + py - 1, xx = x0 + px - 1;
+                float v = 0.f;
+                if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W)
+                    v = static_cast<float>(src[((static_cast<size_t>(n) * p.C + c) * p.H + yy) * p.W + xx]);
+                patch[i] = v;
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");
+            const int sa = ia % NA, ua = ia / NA;
+            if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 4)) break;
+            unsigned char *abase = smem + static_cast<size_t>(sa) * a_stage;
+            for (int row = g; row < MT * kTileM; row += kGatherThreads) {
+                const int ty = row / p.TW, tx = row - ty * p.TW;
+                unsigned char *r_hi = abase + row * 128, *r_lo = r_hi + a_plane;
+                const int sw = row & 7;                          // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+                const float *pp = patch + ty * pw + tx;
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float v2[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int kk = 8 * ch + 2 * e + u;   // compile-time: the loops are fully unrolled
+                            const int c = kk / 9, tap = kk - 9 * c, r = tap / 3, sx = tap - 3 * r;
+                            v2[u] = (c < p.C) ? pp[c * pplane + r * pw + sx] : 0.f;
+                        }
+                        if constexpr (S == 2) {
+                            const __nv_bfloat16 h0 = __float2bfloat16_rn(v2[0]), h1 = __float2bfloat16_rn(v2[1]);
+                            const __nv_bfloat16 l0 = __float2bfloat16_rn(v2[0] - __bfloat162float(h0));
+                            const __nv_bfloat16 l1 = __float2bfloat16_rn(v2[1] - __bfloat162float(h1));
+                            hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+                            lo[e] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
+                        } else {
+                            hi[e] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v2[0]))) |
+                                    (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v2[1]))) << 16);
+                        }
+                    }
+                    *reinterpret_cast<uint4 *>(r_hi + ((ch ^ sw) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    if constexpr (S == 2) *reinterpret_cast<uint4 *>(r_lo + ((ch ^ sw) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy writes -> visible to the MMA
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_fa + 8 * sa) : "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");   // patch free for the next tile
         }
     } else {
         // eight epilogue warps: warp w reads TMEM lanes 32*(w%4).. and one half of the filter columns
@@ -857,7 +924,12 @@ cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t 
 
 template <int BN, int MT, int TERMS, typename T>
 cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
-    auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T>;
+    if (pl.gather) {
+        auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T, true>;
+        if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads + kGatherThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, p);
+    }
+    auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T, false>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
     return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, p);
 }
@@ -968,15 +1040,18 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             const int a_stage = pl.S * (mt * th + hr) * btw * 128;
             const int b_stage = pl.S * pl.BN * 128;
             int na = 2, nb = 2;
-            const int budget = 218 * 1024;
+            // gathered layers stage their fp32 input patch (tile plus border, all channels) behind the rings
+            const int patch = pl.im2col ? ((C * (mt * th + 2) * (btw + 2) * 4 + 1023) / 1024) * 1024 : 0;
+            const int budget = 218 * 1024 - patch;
             while (nb < 6 && na * a_stage + (nb + 1) * b_stage <= budget) ++nb;
             if (na * a_stage + nb * b_stage <= budget) {
                 while (na < 3 && (na + 1) * a_stage + nb * b_stage <= budget) ++na;
                 pl.halo = 1; pl.MT = mt; pl.TW = btw; pl.TH = th; pl.TN = 1;
+                pl.gather = pl.im2col;                           // operand rows built in the kernel, no gathered tensor
                 pl.tiles_x = (W + btw - 1) / btw; pl.tiles_y = (H + mt * th - 1) / (mt * th); pl.tiles_n = N;
                 pl.box_bytes = (mt * th + hr) * btw * 128;
                 pl.na = na; pl.stages = nb;
-                pl.smem_bytes = na * a_stage + nb * b_stage + 1024;
+                pl.smem_bytes = na * a_stage + nb * b_stage + patch + 1024;
                 pl.n_tiles = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
                 pl.grid = std::min(pl.n_tiles, 148);             // persistent CTAs, one per SM
             }

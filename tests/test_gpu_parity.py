@@ -185,8 +185,9 @@ def test_small_stack_with_odd_sizes_and_pools(variants, hw):
     stack.run(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     if variants == ("dense", "dense", "dense"):
-        # one layout kernel for the caller's NCHW input, then three GEMMs: both pools are taken in the epilogues
-        assert B.launch_count() == 4
+        # three GEMMs, both pools taken in their epilogues; the first layer (9*C <= 64) either gathers its operand rows
+        # from the caller's NCHW input itself or has one layout kernel in front
+        assert B.launch_count() in (3, 4)
     assert_close(out.cpu().numpy(), cur, 4 * TOL_F32, f"stack {variants} {hw}")
     stack.free()
     for hd in handles:
