@@ -56,7 +56,7 @@ namespace {
 
 constexpr int kThreads = 320;                // general kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA warp, eight epilogue warps
-constexpr int kGatherThreads = 128;          // plus four gather warps for layers whose operand rows are built in the kernel
+constexpr int kGatherThreads = 256;          // plus eight gather warps for layers whose operand rows are built in the kernel
 constexpr int kTileM = 128;
 constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
 constexpr uint32_t kSpinLimit = 1u << 21;    // bounded mbarrier polling: each poll may block up to ~1 us (hint below)
@@ -787,27 +787,49 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             PATDNN_STAMP(3);
         }
     } else if (GATHER && warp >= kHaloThreads / 32) {
-        // gather warps: per tile (one A stage: KB = 1) they stage the input patch with its one-pixel border in shared
-        // memory (coalesced reads, zeros outside the image), then thread g builds the operand rows g, g+128, ...
-        const T *src = static_cast<const T *>(p.gather_src);
+        // gather warps: the input patch of a tile (all channels, one-pixel border, zeros outside the image) is staged
+        // in shared memory -- double buffered, the next tile's patch is fetched into registers while this tile's rows
+        // are built -- and thread g builds the operand rows g, g+256, ... of the tile's A stage (one stage per tile).
+        const T *__restrict__ src = static_cast<const T *>(p.gather_src);
         const int g = threadIdx.x - kHaloThreads;
-        const int ph = MT * p.TH + 2, pw = p.TW + 2, pplane = ph * pw;
-        float *patch = reinterpret_cast<float *>(smem_b + NB * b_stage);     // [C][ph][pw], behind the two rings
-        int ia = 0;
-        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++ia) {
+        const int ph = MT * p.TH + 2, pw = p.TW + 2, pplane = ph * pw, pcount = p.C * pplane;
+        const int pstride = (pcount + 3) & ~3;
+        float *patch0 = reinterpret_cast<float *>(smem_b + NB * b_stage);    // 2 x [C][ph][pw], behind the two rings
+        constexpr int PF = 8;                                    // patch elements per thread (planner: pcount <= 8 * 256)
+        float pre[PF];
+        auto fetch = [&](int t) {
             int ft, x0, y0, n;
             decode(t, ft, x0, y0, n);
-            for (int i = g; i < p.C * pplane; i += kGatherThreads) {
-                const int c = i / pplane, rem = i - c * pplane, py = rem / pw, px = rem - py * pw;
-                const int yy = y0 + py - 1, xx = x0 + px - 1;
+#pragma unroll
+            for (int u = 0; u < PF; ++u) {
+                const int i = g + u * kGatherThreads;
                 float v = 0.f;
-                if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W)
-                    v = static_cast<float>(src[((static_cast<size_t>(n) * p.C + c) * p.H + yy) * p.W + xx]);
-                patch[i] = v;
+                if (i < pcount) {
+                    const int c = i / pplane, rem = i - c * pplane, py = rem / pw, px = rem - py * pw;
+                    const int yy = y0 + py - 1, xx = x0 + px - 1;
+                    if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W)
+                        v = static_cast<float>(src[((static_cast<size_t>(n) * p.C + c) * p.H + yy) * p.W + xx]);
+                }
+                pre[u] = v;
             }
-            asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");
+        };
+        auto stash = [&](float *dst) {
+#pragma unroll
+            for (int u = 0; u < PF; ++u) {
+                const int i = g + u * kGatherThreads;
+                if (i < pcount) dst[i] = pre[u];
+            }
+        };
+        if (static_cast<int>(blockIdx.x) < n_tiles) { fetch(blockIdx.x); stash(patch0); }
+        asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");
+        int ia = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++ia) {
+            const float *patch = patch0 + (ia & 1) * pstride;
+            const bool more = t + static_cast<int>(gridDim.x) < n_tiles;
+            if (more) fetch(t + gridDim.x);                      // loads in flight while the rows are built
             const int sa = ia % NA, ua = ia / NA;
             if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 4)) break;
+            if (g == 0 && ia == 1) PATDNN_STAMP(11);
             unsigned char *abase = smem + static_cast<size_t>(sa) * a_stage;
             for (int row = g; row < MT * kTileM; row += kGatherThreads) {
                 const int ty = row / p.TW, tx = row - ty * p.TW;
@@ -827,14 +849,14 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                             v2[u] = (c < p.C) ? pp[c * pplane + r * pw + sx] : 0.f;
                         }
                         if constexpr (S == 2) {
-                            const __nv_bfloat16 h0 = __float2bfloat16_rn(v2[0]), h1 = __float2bfloat16_rn(v2[1]);
-                            const __nv_bfloat16 l0 = __float2bfloat16_rn(v2[0] - __bfloat162float(h0));
-                            const __nv_bfloat16 l1 = __float2bfloat16_rn(v2[1] - __bfloat162float(h1));
-                            hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
-                            lo[e] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v2[0], v2[1]);
+                            const float2 hf = __bfloat1622float2(h2);
+                            const __nv_bfloat162 l2 = __floats2bfloat162_rn(v2[0] - hf.x, v2[1] - hf.y);
+                            hi[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                            lo[e] = *reinterpret_cast<const uint32_t *>(&l2);
                         } else {
-                            hi[e] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v2[0]))) |
-                                    (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v2[1]))) << 16);
+                            const __half2 h2 = __floats2half2_rn(v2[0], v2[1]);
+                            hi[e] = *reinterpret_cast<const uint32_t *>(&h2);
                         }
                     }
                     *reinterpret_cast<uint4 *>(r_hi + ((ch ^ sw) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -844,7 +866,10 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy writes -> visible to the MMA
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_fa + 8 * sa) : "memory");
-            asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");   // patch free for the next tile
+            if (g == 0 && ia == 1) PATDNN_STAMP(12);
+            if (more) stash(patch0 + ((ia + 1) & 1) * pstride);
+            asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");   // next patch complete, this one free
+            if (g == 0 && ia == 0) PATDNN_STAMP(9);
         }
     } else {
         // eight epilogue warps: warp w reads TMEM lanes 32*(w%4).. and one half of the filter columns
@@ -1041,13 +1066,14 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             const int b_stage = pl.S * pl.BN * 128;
             int na = 2, nb = 2;
             // gathered layers stage their fp32 input patch (tile plus border, all channels) behind the rings
-            const int patch = pl.im2col ? ((C * (mt * th + 2) * (btw + 2) * 4 + 1023) / 1024) * 1024 : 0;
+            const int pcount = C * (mt * th + 2) * (btw + 2);
+            const int patch = pl.im2col ? ((2 * ((pcount + 3) & ~3) * 4 + 1023) / 1024) * 1024 : 0;   // double buffered
             const int budget = 218 * 1024 - patch;
             while (nb < 6 && na * a_stage + (nb + 1) * b_stage <= budget) ++nb;
             if (na * a_stage + nb * b_stage <= budget) {
                 while (na < 3 && (na + 1) * a_stage + nb * b_stage <= budget) ++na;
                 pl.halo = 1; pl.MT = mt; pl.TW = btw; pl.TH = th; pl.TN = 1;
-                pl.gather = pl.im2col;                           // operand rows built in the kernel, no gathered tensor
+                pl.gather = pl.im2col && pcount <= 8 * 256;      // operand rows built in the kernel, no gathered tensor
                 pl.tiles_x = (W + btw - 1) / btw; pl.tiles_y = (H + mt * th - 1) / (mt * th); pl.tiles_n = N;
                 pl.box_bytes = (mt * th + hr) * btw * 128;
                 pl.na = na; pl.stages = nb;
