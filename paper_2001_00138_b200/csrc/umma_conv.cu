@@ -1057,7 +1057,8 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             const bool fits = 2 * pl.S * (mt_try * th + hr) * tw * 128 + 2 * pl.S * pl.BN * 128 <= 218 * 1024;
             if (fits && u > butil + 1e-9) { butil = u; btw = tw; }
         }
-        if (btw && butil >= util_now - 0.02) {
+        // gathered layers: the MMA work is tiny and the kernel-side gather saves a whole tensor, so padding matters less
+        if (btw && butil >= util_now - (pl.im2col ? 0.30 : 0.02)) {
             const int th = kTileM / btw;
             int mt = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
             if (const char *mv = std::getenv("PATDNN_MT")) mt = (atoi(mv) == 2 && pl.BN == 64) ? 2 : 1;

@@ -108,6 +108,23 @@ def test_resnet_shapes_fp16(i, N):
         assert_close(got, ref, TOL_F16, f"resnet {i} N={N} {variant}")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("shape", [(4, 3, 64, 64, 64), (6, 4, 96, 40, 72), (10, 7, 64, 33, 50), (3, 1, 130, 71, 90)])
+def test_small_channel_layers_gather_their_operand_in_the_kernel(shape, dtype):
+    """9*C <= 64 on the persistent tensor-core kernel: one launch per call (no gathered tensor is written first), image
+    borders, ragged tiles and the zero tail of the 64-deep operand rows included."""
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, C, F, H, W = shape
+    L = synth.make_layer("g", F=F, C=C, N=N, H=H, W=W, seed=4242 + C, n_patterns=8, prune=0.2 if C > 1 else 0.0,
+                         bias_std=0.3, x_dist="normal", dtype=dtype)
+    B.reset_launch_count()
+    got, plan = gpu_layer(L, variant=VARIANTS["dense"])
+    assert plan["variant"] == VARIANTS["dense"]
+    assert B.launch_count() == 1
+    assert_close(got, oracle_layer(L), TOL_F16 if dtype == "f16" else TOL_F32, f"gather {shape} {dtype}")
+
+
 @pytest.mark.parametrize("npat,prune", [(4, 0.0), (6, 0.5), (8, 0.75), (12, 0.9)])
 def test_sweep_points_reduced_batch(npat, prune):
     L = synth.sweep_layer(npat, prune, N=3)
