@@ -155,17 +155,28 @@ def time_oracle_sample(synth, seconds_hint=15.0):
 
 
 def time_layer(h, x, y, stream, torch, reps=20, flush=None):
-    """Mean launch time (us) of one layer call, CUDA events on the launching stream."""
+    """Mean time (us) of one layer call, CUDA events on the launching stream.  Small cases (flush given) replay the call
+    as a one-node-chain CUDA graph: launching from Python costs more than such a layer runs."""
     for _ in range(3):
         h.conv(x, y, stream)
     torch.cuda.synchronize()
+    graph = None
+    if flush is not None:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            h.conv(x, y, torch.cuda.current_stream().cuda_stream)
+        graph.replay()
+        torch.cuda.synchronize()
     tot = 0.0
     for _ in range(reps):
         if flush is not None:
             flush.fill_(1.0)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        h.conv(x, y, stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            h.conv(x, y, stream)
         b.record()
         torch.cuda.synchronize()
         tot += a.elapsed_time(b)
@@ -225,6 +236,12 @@ def run_suite(args):
                 measure("sweep", L, 64, order=synth.random_filter_order(512, 7))
                 measure("sweep", L, 64, variant="tiled")
                 measure("sweep", L, 64, variant="tiled", order=synth.random_filter_order(512, 7))
+    if "cifar" in which or "all" in which:
+        suite_cifar_stack(B, synth, torch, hbm, stream)
+    if "storage" in which or "all" in which:
+        suite_storage(B, synth)
+    if "context" in which or "all" in which:
+        suite_dense_context(synth, torch)
     if "ablation" in which or "all" in which:
         seen = set()
         for i in range(13):
@@ -234,6 +251,106 @@ def run_suite(args):
             L = synth.vgg16_layer(i, N=1)
             for variant in ("noopt", "reorder", "tiled", "dense_tc"):
                 measure("ablation_vgg_unique_layers", L, 1, variant=variant, reps=5 if variant in ("noopt", "reorder") else 20)
+
+
+def suite_cifar_stack(B, synth, torch, hbm, stream):
+    """VGG-16's conv stack on a CIFAR-sized 32x32 input (the paper's second dataset): 32,32,16,16,8,8,8,4,4,4,2,2,2."""
+    for N in (1, 32, 256):
+        layers = [synth.vgg16_layer(i, N=N, spatial_scale=7) for i in range(13)]
+        handles = [B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, relu=True, bias=L.bias) for L in layers]
+        pools = [1 if i in synth.VGG16_POOL_AFTER else 0 for i in range(13)]
+        stack = B.Stack(handles, pools)
+        x = torch.from_numpy(synth.vgg16_input(N, 7)).cuda()
+        out = torch.empty(stack.out_shape(), device="cuda")
+        graph = torch.cuda.CUDAGraph()
+        stack.run(x, out, stream)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph):
+            stack.run(x, out, torch.cuda.current_stream().cuda_stream)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        a.record()
+        for _ in range(reps):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / reps * 1e3
+        for h in handles:
+            h.check()
+        costs = [layer_costs(L, hbm) for L in layers]
+        flops, roof = sum(c[0] for c in costs), sum(c[2] for c in costs)
+        print(json.dumps({"suite": "cifar_vgg16_stack", "batch": N, "us": round(us, 1),
+                          "gflops_nonzero": round(flops / us / 1e3, 1), "roofline_us": round(roof, 1),
+                          "frac": round(roof / us, 3),
+                          "kernels": "".join({3: "t", 4: "D"}.get(h.plan()["variant"], "g") for h in handles),
+                          "timing": "CUDA-graph replay of the chained stack, working set L2-resident"}), flush=True)
+        stack.free()
+        for h in handles:
+            h.free()
+
+
+def suite_storage(B, synth):
+    """Index and total bytes of the FKW arrays against CSR over the same weights (Section 6.4's comparison), from the
+    arrays the encoder really emits; overall rates 8x / 12x / 18x = 4-of-9 patterns times connectivity pruning."""
+    for rate in (8, 12, 18):
+        keep = 9.0 / (4.0 * rate)
+        for (C, F) in ((256, 256), (512, 512)):
+            L = synth.make_layer(f"storage_c{C}f{F}_{rate}x", F=F, C=C, N=1, H=14, W=14, seed=6000 + rate, n_patterns=8,
+                                 prune=1.0 - keep, draw_input=False)
+            h = B.encode(L.weights, L.mask, L.patterns, N=1, H=14, W=14, host_only=True)
+            a = h.export()
+            K = int(a["index"].shape[0])
+            nnz = 4 * K
+            fkw_idx32 = 4 * (a["offset"].size + a["reorder"].size + a["index"].size + a["stride"].size)
+            fkw_idx16 = 2 * a["index"].size + 4 * a["offset"].size + 2 * a["reorder"].size + 2 * a["stride"].size
+            csr_idx32 = 4 * (F + 1) + 4 * nnz
+            csr_idx16 = 4 * (F + 1) + 2 * nnz
+            w_bytes = 4 * nnz
+            print(json.dumps({"suite": "storage_fkw_vs_csr", "layer": L.name, "overall_rate": rate, "kernels_kept": K,
+                              "weights_bytes": w_bytes, "fkw_index_bytes_i32": fkw_idx32, "csr_index_bytes_i32": csr_idx32,
+                              "fkw_index_bytes_u16": fkw_idx16, "csr_index_bytes_u16": csr_idx16,
+                              "index_saving_i32": round(1 - fkw_idx32 / csr_idx32, 4),
+                              "total_saving_i32": round(1 - (fkw_idx32 + w_bytes) / (csr_idx32 + w_bytes), 4),
+                              "total_saving_u16": round(1 - (fkw_idx16 + w_bytes) / (csr_idx16 + w_bytes), 4)}), flush=True)
+            h.free()
+
+
+def suite_dense_context(synth, torch):
+    """Library context, not a target: torch's dense conv2d (cuDNN, fp32 without TF32) on the unpruned shape of each
+    unique VGG layer, next to which the pattern-sparse numbers of the headline run can be read."""
+    import torch.nn.functional as Fn
+    torch.backends.cudnn.allow_tf32 = False
+    torch.backends.cuda.matmul.allow_tf32 = False
+    flush = torch.empty(256 * 1024 * 1024 // 4, device="cuda")
+    for N in (1, 32):
+        seen = set()
+        for i in range(13):
+            if synth.VGG16_CONVS[i] in seen:
+                continue
+            seen.add(synth.VGG16_CONVS[i])
+            C, F, S = synth.VGG16_CONVS[i]
+            x = torch.rand((N, C, S, S), device="cuda")
+            w = torch.randn((F, C, 3, 3), device="cuda") * 0.05
+            for _ in range(3):
+                Fn.conv2d(x, w, padding=1)
+            torch.cuda.synchronize()
+            tot, reps = 0.0, 10
+            for _ in range(reps):
+                if N == 1:
+                    flush.fill_(1.0)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                Fn.conv2d(x, w, padding=1)
+                b.record()
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+            us = tot / reps * 1e3
+            print(json.dumps({"suite": "dense_conv2d_context", "layer": f"c{C}f{F}_{S}", "batch": N, "us": round(us, 1),
+                              "dense_gflops": round(2.0 * 9 * C * F * S * S * N / us / 1e3, 1),
+                              "library": "torch.nn.functional.conv2d (cuDNN), fp32, TF32 off"}), flush=True)
 
 
 def run_reference(args):
@@ -273,7 +390,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
-    ap.add_argument("--suite", default="", help="instead of the headline step: cfg2,resnet,sweep,ablation or all "
+    ap.add_argument("--suite", default="", help="instead of the headline step: cfg2,resnet,sweep,ablation,cifar,storage,context or all "
                                                 "(one JSON line per measured point)")
     args = ap.parse_args()
     if args.impl == "reference":

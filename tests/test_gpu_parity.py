@@ -136,13 +136,14 @@ def test_sweep_points_reduced_batch(npat, prune):
     assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune} random filter order")
 
 
-def test_vgg_stack_reduced_spatial_per_layer_and_chained():
-    """All 13 layers at 1/4 spatial size, batch 2: each GPU layer is fed the oracle's input for that layer
-    (binding check), and the chained GPU stack is compared with the chained oracle."""
+@pytest.mark.parametrize("scale,N", [(4, 2), (7, 5)])
+def test_vgg_stack_reduced_spatial_per_layer_and_chained(scale, N):
+    """All 13 layers at 1/4 spatial size (56x56 input) and at 1/7 (the 32x32 input of the CIFAR-sized network, down to
+    2x2 images): each GPU layer is fed the oracle's input for that layer (binding check), and the chained GPU stack is
+    compared with the chained oracle."""
     import oracle
     import torch
     from paper_2001_00138_b200 import binding as B
-    scale, N = 4, 2
     x = synth.vgg16_input(N, scale)
     layers, handles = [], []
     cur = x
