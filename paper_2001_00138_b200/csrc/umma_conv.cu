@@ -574,6 +574,8 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         // both barriers, also after a timed-out wait, so nobody is left waiting.
         const int cols = BN / ks;
         const uint32_t rbase = smem_u32(smem);
+        __syncwarp();                                           // lane 0 of the two role warps rejoins its warp: the
+                                                                // cluster barriers below are warp-aligned instructions
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
         if (threadIdx.x == 64) PATDNN_STAMP(7);
         if (acc_ready) {
