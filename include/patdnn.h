@@ -179,7 +179,10 @@ typedef struct {
     int32_t warps_per_cta;
     int32_t channels_per_stage; /* input channels staged per shared-memory buffer */
     int32_t channel_splits;     /* >1: the channel range is split across a thread-block cluster */
-    int32_t grid_x, grid_y, grid_z;
+    int32_t grid_x, grid_y, grid_z; /* CUDA-core kernels: the launch grid.  Tensor-core path: grid_x = CTAs of the main
+                                     * launch (= tiles for the one-tile-per-CTA kernel), grid_y = tiles shared by the
+                                     * persistent CTAs (1 otherwise), grid_z = 1 + tiles handed to a second, K-split
+                                     * launch when the tile count is not a whole number of 148-CTA rounds */
     int32_t smem_bytes;
     int64_t device_bytes;       /* bytes of the private device layout */
     int64_t entries;            /* kernel entries in the device layout (kept kernels plus padding) */

@@ -117,7 +117,7 @@ static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const pat
 #endif
     cudaError_t e = launch_dense_gemm(pl, p, h->desc.dtype, st);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core kernel launch");
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    g_launches.fetch_add(pl.tail_tiles ? 2 : 1, std::memory_order_relaxed);
     return PATDNN_OK;
 }
 
@@ -410,7 +410,10 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         const DensePlan &p = h->dense;
         info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 10;
         info->channels_per_stage = 64; info->channel_splits = p.ksplit;
-        info->grid_x = p.grid; info->grid_y = p.halo ? p.n_tiles : 1; info->grid_z = 1; info->smem_bytes = p.smem_bytes;
+        // grid_x: CTAs of the main launch (plus, for the one-tile-per-CTA kernel, the tiles of a K-split tail launch, so
+        // that it stays the tile count); grid_y: tiles shared by the persistent CTAs; grid_z: tiles given to a tail launch
+        info->grid_x = p.halo ? p.grid : p.grid + p.tail_tiles; info->grid_y = p.halo ? p.n_tiles : 1;
+        info->grid_z = 1 + p.tail_tiles; info->smem_bytes = p.smem_bytes;
         info->entries = static_cast<int64_t>(p.taps) * p.Fp * p.Cp;
     } else {
         info->tile_rows = 1; info->tile_cols = 1; info->filters_per_warp = 1; info->warps_per_cta = 8;

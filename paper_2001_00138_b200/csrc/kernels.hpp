@@ -136,6 +136,10 @@ struct DensePlan {
     int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
     int gather = 0;                        // im2col layer on the persistent kernel: operand rows gathered in the kernel
+    // Tail of a grid that is not a whole number of 148-CTA rounds: the last tail_tiles tiles run as a second launch of
+    // the one-tile-per-CTA kernel with the K loop split tail_ks ways (clusters), instead of costing a whole extra round.
+    int tail_tiles = 0, tail_ks = 1, tail_stages = 0, tail_smem = 0, tail_box_bytes = 0;
+    CUtensorMap mapA_tail{};               // per-tap box of the tail launch (no halo rows)
     int poolable = 0;                      // boxes meet the conditions of the fused max-pool epilogue (mode 4)
     CUtensorMap mapA{}, mapB{};
 };
@@ -151,6 +155,8 @@ struct DenseParams {
     int mode;                   // 0: out = caller's NCHW tensor; 3: out = next layer's split [S][N][H][W][out_cp] buffer;
                                 // 4: as 3 after a fused 2x2 max-pool, [S][N][H/2][W/2][out_cp] (needs a pool_tiles plan)
     int out_cp;                 // channel pitch of the mode-3/4 destination
+    int tile_base;              // one-tile-per-CTA kernel: index of the first tile this launch covers
+    int tile_limit;             // persistent kernel: tiles [0, tile_limit) only (0 = all)
     const void *gather_src;     // gather plans: the layer's NCHW input (fp32 or fp16 as the layer's dtype)
 };
 

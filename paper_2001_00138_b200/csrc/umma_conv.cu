@@ -449,7 +449,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     // iterations -- into ks ranges; then the filter tile index is fastest so that CTAs sharing a pixel box run together.
     const int ks = p.ksplit;
     const int rank = blockIdx.x % ks;
-    int pt = blockIdx.x / ks;
+    int pt = blockIdx.x / ks + p.tile_base;
     const int ft = pt % p.n_ftiles; pt /= p.n_ftiles;
     const int tix = pt % p.tiles_x; pt /= p.tiles_x;
     const int tiy = pt % p.tiles_y; pt /= p.tiles_y;
@@ -664,7 +664,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                    bar_eb = smem_u32(&bars[24]), bar_af = smem_u32(&bars[32]), bar_ae = smem_u32(&bars[34]);
     int *status = p.status;
     const int row_bytes = p.TW * 128;
-    const int n_tiles = p.n_ftiles * p.tiles_x * p.tiles_y * p.tiles_n;
+    const int n_tiles = p.tile_limit > 0 ? p.tile_limit : p.n_ftiles * p.tiles_x * p.tiles_y * p.tiles_n;
     const int KB = p.KB;
     const int nshift = p.taps == 9 ? 3 : 1;                     // 3 horizontal shifts x 3 vertical taps, or one gathered tap
 
@@ -942,11 +942,24 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// The tail launch of a plan: its last tail_tiles tiles on the one-tile-per-CTA kernel, K loop split over clusters.
+template <int BN, int TERMS, typename T>
+cudaError_t launch_tail(const DensePlan &pl, const DenseParams &p, cudaStream_t st, int first_tile) {
+    DenseParams q = p;
+    q.tile_base = first_tile; q.tile_limit = 0;
+    q.ksplit = pl.tail_ks; q.stages = pl.tail_stages; q.box_bytes = pl.tail_box_bytes;
+    q.iters_per_split = (pl.taps * pl.KB + pl.tail_ks - 1) / pl.tail_ks;
+    return launch_pdl(conv_umma_kernel<BN, TERMS, T>, dim3(pl.tail_tiles * pl.tail_ks), dim3(kThreads), pl.tail_smem, st,
+                      pl.tail_ks, pl.mapA_tail, pl.mapB, q);
+}
+
 template <int BN, int TERMS, typename T>
 cudaError_t launch_umma(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
     auto kern = conv_umma_kernel<BN, TERMS, T>;
     if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-    return launch_pdl(kern, dim3(pl.grid), dim3(kThreads), pl.smem_bytes, st, pl.ksplit, pl.mapA, pl.mapB, p);
+    cudaError_t e = launch_pdl(kern, dim3(pl.grid), dim3(kThreads), pl.smem_bytes, st, pl.ksplit, pl.mapA, pl.mapB, p);
+    if (e == cudaSuccess && pl.tail_tiles) e = launch_tail<BN, TERMS, T>(pl, p, st, pl.grid);
+    return e;
 }
 
 template <int BN, int MT, int TERMS, typename T>
@@ -957,8 +970,17 @@ cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t 
         return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads + kGatherThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, p);
     }
     auto kern = conv_umma_halo_kernel<BN, MT, TERMS, T, false>;
-    if (prep) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-    return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, p);
+    if (prep) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        if (e == cudaSuccess && pl.tail_tiles)
+            e = cudaFuncSetAttribute(conv_umma_kernel<BN, TERMS, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        return e;
+    }
+    DenseParams q = p;
+    q.tile_limit = pl.tail_tiles ? pl.n_tiles - pl.tail_tiles : 0;
+    cudaError_t e = launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, q);
+    if (e == cudaSuccess && pl.tail_tiles) e = launch_tail<BN, TERMS, T>(pl, p, st, pl.n_tiles - pl.tail_tiles);
+    return e;
 }
 
 cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
@@ -1086,6 +1108,27 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             }
         }
     }
+    // Round quantisation: T equal tiles on 148 SMs take ceil(T/148) rounds.  When the last round is nearly empty its
+    // tiles go to a second launch whose K loop is split over clusters (largest split that still fits one wave).
+    const char *tv = std::getenv("PATDNN_TAIL");
+    const int T = pl.halo ? pl.n_tiles : pl.grid;
+    if (!(tv && tv[0] == '0') && pl.ksplit == 1 && pl.MT == 1 && !pl.gather && T > 148 && T % 148 != 0) {
+        const int tail = T % 148;
+        int tks = 0;
+        for (int cand : {8, 4, 2}) {
+            const int cap = cand == 8 ? 120 : (cand == 4 ? 132 : 148);
+            if (tail * cand <= cap && total_iters / cand >= 2 && pl.BN / cand >= 8) { tks = cand; break; }
+        }
+        if (tks) {
+            pl.tail_tiles = tail; pl.tail_ks = tks;
+            const int tstage = pl.S * (kTileM * 128 + pl.BN * 128);
+            pl.tail_stages = std::max(2, std::min(8, (220 * 1024) / tstage));
+            pl.tail_smem = pl.tail_stages * tstage + 1024;
+            pl.tail_box_bytes = pl.TW * pl.TH * pl.TN * 128;
+            if (pl.halo) pl.grid = std::min(T - tail, 148);
+            else pl.grid = T - tail;
+        }
+    }
 }
 
 // Dense split weights [S][9][Fp][Cp] (16-bit words) from the canonical FKW arrays.
@@ -1130,6 +1173,16 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
                              (cuuint32_t)pl.TN, 1};
         cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (enc(&pl.mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    if (pl.tail_tiles) {
+        cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)pl.S};
+        cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)W * pl.Cp * 2, (cuuint64_t)H * W * pl.Cp * 2,
+                                 (cuuint64_t)N * H * W * pl.Cp * 2};
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)pl.TH, (cuuint32_t)pl.TN, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (enc(&pl.mapA_tail, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return PATDNN_E_CUDA;
     }
