@@ -80,6 +80,8 @@ struct patdnn_layer {
 struct patdnn_stack_s {
     std::vector<patdnn_handle> layers;
     std::vector<int32_t> pool;
+    std::vector<int> smallc;                  // per layer: index into smallc_w, or -1
+    std::vector<SmallCWeights> smallc_w;      // few-channel layers fused with the layout of the tensor-core layer after them
     void *buf[2] = {nullptr, nullptr};
     void *d_in = nullptr, *d_out = nullptr;   // staging buffers of patdnn_stack_run_host
     size_t buf_bytes = 0, in_bytes = 0, out_bytes = 0;
@@ -476,6 +478,19 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         h->dense_pool = pp;
         h->dense_pool_state = 1;
     }
+    // CUDA-core layer with few input channels -> tensor-core layer (no pool between): one kernel that writes the second
+    // layer's operands instead of an NCHW tensor plus a layout pass
+    s->smallc.assign(n, -1);
+    for (int i = 0; i + 1 < n; ++i) {
+        patdnn_layer *h = s->layers[i], *nx = s->layers[i + 1];
+        const patdnn_desc &d = h->desc;
+        if (h->variant == PATDNN_VARIANT_DENSE_TC || s->pool[i] || nx->variant != PATDNN_VARIANT_DENSE_TC || nx->dense.im2col ||
+            nx->dense.Cp != 64 || !smallc_split_supported(d.F, d.C) || std::getenv("PATDNN_NO_SMALLC"))
+            continue;
+        s->smallc_w.emplace_back();
+        build_smallc_weights(h->fkw, h->bias, s->smallc_w.back());
+        s->smallc[i] = static_cast<int>(s->smallc_w.size()) - 1;
+    }
     s->oN = N; s->oF = C; s->oH = H; s->oW = W;
     s->buf_bytes = std::max<size_t>(max_bytes, 16);
     const patdnn_desc &d0 = handles[0]->desc;
@@ -544,6 +559,17 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
                 if (rc) return rc;
                 cur = s->buf[which];
                 which ^= 1;
+            }
+            if (s->smallc[i] >= 0) {
+                patdnn_layer *nx = s->layers[i + 1];
+                cudaError_t e = launch_smallc_split(s->smallc_w[s->smallc[i]], cur, d.dtype == PATDNN_F16, nx->d_act, d.N, d.C, d.H,
+                                                    d.W, d.F, d.relu, nx->dense.Cp, nx->dense.S, st);
+                if (e != cudaSuccess) return cuda_fail(e, "few-channel kernel launch");
+                g_launches.fetch_add(1, std::memory_order_relaxed);
+                direct = true;
+                cur_pool = false;
+                curH = d.H; curW = d.W;
+                continue;
             }
             void *dst = (last && !s->pool[i]) ? out : s->buf[which];
             const int rc = patdnn_conv(h, cur, dst, stream);

@@ -163,6 +163,18 @@ struct DenseParams {
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static
 int static_scratch_address(void **ptr);                    // PATDNN_* status; first call per device looks the address up
 
+// ---- first-layer kernel writing a tensor-core layer's operands (smallc_split.cu) ----------------------------------
+constexpr int kSmallCTaps = 36;            // 9 taps x at most 4 input channels
+struct SmallCWeights {                     // passed by value as a kernel parameter: weights become constant-bank operands
+    float w[64 * kSmallCTaps];             // [filter][9*c + tap], zeros where the pattern keeps nothing
+    float bias[64];
+};
+bool smallc_split_supported(int F, int C);
+void build_smallc_weights(const Fkw &fkw, const std::vector<float> &bias, SmallCWeights &wt);
+// in: NCHW (fp32 or fp16); dst: [S][N][H][W][Cp] split operands of the next layer (Cp = 64), bias + ReLU applied.
+cudaError_t launch_smallc_split(const SmallCWeights &wt, const void *in, int in_is_half, void *dst, int N, int C, int H, int W,
+                                int F, int relu, int Cp, int S, cudaStream_t st);
+
 bool dense_supported(int F, int C, int N, int H, int W);
 // pool_tiles: only pixel boxes whose epilogue can max-pool in registers (one image per box, 2/4/8/16 pixels wide, starting
 // on even rows); sets pl.poolable.  force_bn pins the filter tile width, so that a second plan of a layer shares the

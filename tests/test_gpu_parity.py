@@ -125,6 +125,38 @@ def test_small_channel_layers_gather_their_operand_in_the_kernel(shape, dtype):
     assert_close(got, oracle_layer(L), TOL_F16 if dtype == "f16" else TOL_F32, f"gather {shape} {dtype}")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("shape", [(3, 3, 64, 13, 9), (2, 1, 40, 32, 32), (1, 4, 64, 7, 50), (5, 2, 17, 6, 6)])
+def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype):
+    """CUDA-core layer with C <= 4 and F <= 64 followed by a tensor-core layer: the stack runs ONE kernel for the first
+    layer that writes the second layer's split operands (no NCHW tensor, no layout kernel), then the GEMM."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, C, F, H, W = shape
+    dt = B.F16 if dtype == "f16" else B.F32
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    L0 = synth.make_layer("f0", F=F, C=C, N=N, H=H, W=W, seed=77 + C, prune=0.0, bias_std=0.3, x_dist="normal", dtype=dtype)
+    L1 = synth.make_layer("f1", F=48, C=F, N=N, H=H, W=W, seed=78 + C, prune=0.5, bias_std=0.3, draw_input=False, dtype=dtype,
+                          w_std=0.2)
+    h0 = B.encode(L0.weights, L0.mask, L0.patterns, N=N, H=H, W=W, dtype=dt, relu=True, bias=L0.bias, variant=VARIANTS["reorder"])
+    h1 = B.encode(L1.weights, L1.mask, L1.patterns, N=N, H=H, W=W, dtype=dt, relu=False, bias=L1.bias, variant=VARIANTS["dense"])
+    mid = oracle.conv3x3(L0.x, L0.weights, L0.mask, L0.bias, True)
+    if dtype == "f16":
+        mid = mid.astype(np.float16).astype(np.float32)          # the layer boundary stores fp16
+    ref = oracle.conv3x3(mid, L1.weights, L1.mask, L1.bias, False)
+    stack = B.Stack([h0, h1], [0, 0])
+    out = torch.empty((N, 48, H, W), device="cuda", dtype=tdt)
+    B.reset_launch_count()
+    stack.run(torch.from_numpy(L0.x).to("cuda", dtype=tdt), out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert B.launch_count() == 2
+    assert_close(out.float().cpu().numpy(), ref, 3 * (TOL_F16 if dtype == "f16" else TOL_F32), f"fused first layer {shape} {dtype}")
+    stack.free()
+    h0.free()
+    h1.free()
+
+
 @pytest.mark.parametrize("npat,prune", [(4, 0.0), (6, 0.5), (8, 0.75), (12, 0.9)])
 def test_sweep_points_reduced_batch(npat, prune):
     L = synth.sweep_layer(npat, prune, N=3)
