@@ -48,7 +48,11 @@ __device__ __forceinline__ void trace_stamp(int slot) {
     if (blockIdx.x < (1 << 12)) g_trace[blockIdx.x * 16 + slot] = t;
 }
 #define PATDNN_STAMP(slot) trace_stamp(slot)
+#define PATDNN_TIMED(acc, expr) [&] { const long long t__ = clock64(); const bool r__ = (expr); (acc) += clock64() - t__; return r__; }()
+#define PATDNN_PUT(slot, v) do { if (blockIdx.x < (1 << 12)) g_trace[blockIdx.x * 16 + (slot)] = (unsigned long long)(v); } while (0)
 #else
+#define PATDNN_TIMED(acc, expr) (expr)
+#define PATDNN_PUT(slot, v)
 #define PATDNN_STAMP(slot)
 #endif
 
@@ -737,21 +741,22 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
             int ia = 0, ib = 0, j = 0;
             bool ok = true;
+            [[maybe_unused]] long long w_fa = 0, w_fb = 0, w_ae = 0;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
                 const int buf = j & 1, ub2 = j >> 1;
-                if (ub2 > 0 && !mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2)) { ok = false; break; }
+                if (ub2 > 0 && !PATDNN_TIMED(w_ae, mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2))) { ok = false; break; }
                 tc_fence_after();
                 bool first = true;
                 for (int cb = 0; cb < KB && ok; ++cb) {
                     for (int sx = 0; sx < nshift && ok; ++sx) {
                         const int sa = ia % NA, ua = ia / NA;
-                        ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
+                        ok = PATDNN_TIMED(w_fa, mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2));
                         if (!ok) break;
                         if (ia == 0) PATDNN_STAMP(2);
                         const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
                         for (int r = 0; r < nshift && ok; ++r) {
                             const int sb = ib % NB, ub = ib / NB;
-                            ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
+                            ok = PATDNN_TIMED(w_fb, mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2));
                             if (!ok) break;
                             tc_fence_after();
                             const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
@@ -787,6 +792,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 if (ok) umma_commit(bar_af + 8 * buf);
             }
             PATDNN_STAMP(3);
+            PATDNN_PUT(13, w_fa); PATDNN_PUT(14, w_fb); PATDNN_PUT(15, w_ae);
         }
     } else if (GATHER && warp >= kHaloThreads / 32) {
         // gather warps: the input patch of a tile (all channels, one-pixel border, zeros outside the image) is staged
