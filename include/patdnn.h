@@ -195,7 +195,9 @@ PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
  * max-pool (the VGG-16 arrangement).  The stack owns two ping-pong activation buffers; the handles stay owned by
  * the caller and must outlive the stack.  Between two tensor-core layers no NCHW tensor is formed: the first one's
  * kernel writes the second one's operands (after the pool, where one follows, for which patdnn_stack_create may add a
- * second launch plan to the first layer's handle).  A handle may serve several stacks, but not two calls that overlap
+ * second launch plan to the first layer's handle); a first layer with at most 4 input channels and 64 filters that is
+ * followed by a tensor-core layer runs as one FP32 kernel that writes that layer's operands.  A handle may serve
+ * several stacks, but not two calls that overlap
  * on the GPU: its operand buffer is shared.
  *   patdnn_stack_create   handles HOST [n]; pool_after HOST [n] (1 = max-pool after that layer) or NULL
  *   patdnn_stack_run      in DEVICE [N][C0][H0][W0]; out DEVICE, the last layer's (pooled) output; asynchronous
