@@ -570,9 +570,9 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     if (ks > 1) {
         // Sum the K ranges across the cluster through distributed shared memory.  CTA r finishes the columns
         // [r*BN/ks, (r+1)*BN/ks): every CTA PUSHES the matching slice of its partial tile into r's shared memory
-        // (remote stores need no answer, remote loads would expose their latency; a warp stores 128 contiguous bytes --
-        // 16-byte stores scattered at a row pitch measured twice as slow), slot = sender's rank, layout
-        // [slot][column][pixel]; then r adds
+        // (remote stores need no answer, remote loads would expose their latency; a warp's 16-byte stores cover 512
+        // contiguous bytes -- the same stores scattered at a row pitch measured twice as slow as 4-byte ones), slot =
+        // sender's rank, layout [slot][column quad][pixel][4]; then r adds
         // the ks slots in rank order from its own memory.  Barrier 1: every CTA's MMAs have read their pipeline
         // buffers, which the slots reuse.  Barrier 2: all slots have landed.  Every thread of every CTA takes part in
         // both barriers, also after a timed-out wait, so nobody is left waiting.
@@ -593,11 +593,16 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     const int owner = (c0 + j0) / cols, cl = (c0 + j0) - owner * cols;
                     uint32_t remote;
                     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(rbase), "r"(owner));
-                    remote += ((rank * cols + cl) * kTileM + m) * 4;
+                    // slot layout [sender][column quad][pixel][4 columns]: a warp's 16-byte stores are 512 contiguous bytes
+                    remote += (((rank * cols + cl) >> 2) * kTileM + m) * 16;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float val = __uint_as_float(v[j0 + j]) + (MERGE ? __uint_as_float(v2[j0 + j]) : 0.f);
-                        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote + j * kTileM * 4), "f"(val) : "memory");
+                    for (int h4 = 0; h4 < 2; ++h4) {
+                        float w4[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            w4[j] = __uint_as_float(v[j0 + 4 * h4 + j]) + (MERGE ? __uint_as_float(v2[j0 + 4 * h4 + j]) : 0.f);
+                        asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote + h4 * kTileM * 16), "f"(w4[0]),
+                                     "f"(w4[1]), "f"(w4[2]), "f"(w4[3]) : "memory");
                     }
                 }
             }
@@ -606,16 +611,19 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
         if (threadIdx.x == 64) PATDNN_STAMP(9);
         if (warp >= 2) {
-            const float *R = reinterpret_cast<const float *>(smem);
+            const float4 *R4 = reinterpret_cast<const float4 *>(smem);
             const int cbeg = rank * cols;
 #pragma unroll 1
             for (int c0 = 8 * half; c0 < cols; c0 += 16) {
                 float a[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) a[j] = 0.f;
-                for (int qq = 0; qq < ks; ++qq)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) a[j] += R[(qq * cols + c0 + j) * kTileM + m];
+                for (int qq = 0; qq < ks; ++qq) {
+                    const float4 lo4 = R4[((qq * cols + c0) >> 2) * kTileM + m];
+                    const float4 hi4 = R4[(((qq * cols + c0) >> 2) + 1) * kTileM + m];
+                    a[0] += lo4.x; a[1] += lo4.y; a[2] += lo4.z; a[3] += lo4.w;
+                    a[4] += hi4.x; a[5] += hi4.y; a[6] += hi4.z; a[7] += hi4.w;
+                }
                 emit_chunk<8, T>(p, a, s_bias + cbeg + c0, f0 + cbeg + c0, n, y, x, pix_ok);
             }
         }
