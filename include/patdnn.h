@@ -202,12 +202,21 @@ PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
  *   patdnn_stack_create   handles HOST [n]; pool_after HOST [n] (1 = max-pool after that layer) or NULL
  *   patdnn_stack_run      in DEVICE [N][C0][H0][W0]; out DEVICE, the last layer's (pooled) output; asynchronous
  *   patdnn_stack_run_host the same with HOST buffers; copies in, runs, copies out, waits for the stream
+ *   patdnn_stack_submit_host / patdnn_stack_wait_host  the pipelined form of run_host for a stream of batches: submit
+ *                         enqueues copy-in (library-owned copy stream), the kernels (caller's stream) and copy-out
+ *                         (second copy stream) and returns; wait blocks until the OLDEST submitted batch has landed in
+ *                         its out_host.  At most two batches may be in flight (a third submit returns E_STACK);
+ *                         in_host must stay untouched until the kernels of its batch ran, i.e. until its wait;
+ *                         pinned host memory is needed for the copies to overlap.  All submits of a stack must use
+ *                         the same stream.
  *   patdnn_stack_out_shape  N, F, H, W of the stack's output
  * Errors: E_NULL, E_STACK, E_CUDA, E_NO_DEVICE.
  */
 PATDNN_API int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after, int32_t n, patdnn_stack *out);
 PATDNN_API int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream);
 PATDNN_API int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
+PATDNN_API int patdnn_stack_submit_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
+PATDNN_API int patdnn_stack_wait_host(patdnn_stack s);
 PATDNN_API int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, int32_t *W);
 PATDNN_API int patdnn_stack_free(patdnn_stack s);
 

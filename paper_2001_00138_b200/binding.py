@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "OK", 1: "E_NULL", 2: "E_SHAPE", 3: "E_PATTERN_SET", 4: "E_MA
 EXPORTED_SYMBOLS = (
     "patdnn_encode", "patdnn_conv", "patdnn_conv_static", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
-    "patdnn_stack_free", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
+    "patdnn_stack_free", "patdnn_stack_submit_host", "patdnn_stack_wait_host", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
     "patdnn_last_cuda_error", "patdnn_version",
 )
 
@@ -84,6 +84,8 @@ def load() -> ctypes.CDLL:
     lib.patdnn_stack_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(i32), i32, ctypes.POINTER(vp)]
     lib.patdnn_stack_run.argtypes = [vp, vp, vp, vp]
     lib.patdnn_stack_run_host.argtypes = [vp, vp, vp, vp]
+    lib.patdnn_stack_submit_host.argtypes = [vp, vp, vp, vp]
+    lib.patdnn_stack_wait_host.argtypes = [vp]
     lib.patdnn_stack_out_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 4
     lib.patdnn_stack_free.argtypes = [vp]
     lib.patdnn_maxpool2x2.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
@@ -244,6 +246,14 @@ class Stack:
     def run_host(self, x: np.ndarray, out: np.ndarray, stream: int = 0) -> None:
         assert x.flags.c_contiguous and out.flags.c_contiguous
         _check(load().patdnn_stack_run_host(self._h, x.ctypes.data, out.ctypes.data, stream), "patdnn_stack_run_host")
+
+    def submit_host(self, x: np.ndarray, out: np.ndarray, stream: int = 0) -> None:
+        """Pipelined run_host: returns at once; at most two batches in flight; pair every call with wait_host()."""
+        assert x.flags.c_contiguous and out.flags.c_contiguous
+        _check(load().patdnn_stack_submit_host(self._h, x.ctypes.data, out.ctypes.data, stream), "patdnn_stack_submit_host")
+
+    def wait_host(self) -> None:
+        _check(load().patdnn_stack_wait_host(self._h), "patdnn_stack_wait_host")
 
     def free(self) -> None:
         if self._h:

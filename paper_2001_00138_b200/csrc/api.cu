@@ -80,6 +80,11 @@ struct patdnn_layer {
 struct patdnn_stack_s {
     std::vector<patdnn_handle> layers;
     std::vector<int32_t> pool;
+    // pipelined host entry point: two input/output slots, one stream per copy direction
+    void *p_in[2] = {nullptr, nullptr}, *p_out[2] = {nullptr, nullptr};
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_run[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    int64_t submitted = 0, waited = 0;
     std::vector<int> smallc;                  // per layer: index into smallc_w, or -1
     std::vector<SmallCWeights> smallc_w;      // few-channel layers fused with the layout of the tensor-core layer after them
     void *buf[2] = {nullptr, nullptr};
@@ -603,6 +608,45 @@ int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *out_host, v
     return PATDNN_OK;
 }
 
+// Pipelined variant of patdnn_stack_run_host: the copies of call i+1 overlap the kernels of call i.
+int patdnn_stack_submit_host(patdnn_stack s, const void *in_host, void *out_host, void *stream) {
+    if (!s || !in_host || !out_host) return PATDNN_E_NULL;
+    if (s->submitted - s->waited >= 2) return PATDNN_E_STACK;            // both slots in flight: wait for one first
+    if (!s->h2d) {
+        CU(cudaStreamCreateWithFlags(&s->h2d, cudaStreamNonBlocking));
+        CU(cudaStreamCreateWithFlags(&s->d2h, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            CU(cudaMalloc(&s->p_in[b], std::max<size_t>(s->in_bytes, 16)));
+            CU(cudaMalloc(&s->p_out[b], std::max<size_t>(s->out_bytes, 16)));
+            CU(cudaEventCreateWithFlags(&s->ev_in[b], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&s->ev_run[b], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&s->ev_out[b], cudaEventDisableTiming));
+        }
+    }
+    const int b = static_cast<int>(s->submitted & 1);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // slot b was last used two submissions ago and has been waited for (checked above), so its buffers are free
+    CU(cudaMemcpyAsync(s->p_in[b], in_host, s->in_bytes, cudaMemcpyHostToDevice, s->h2d));
+    CU(cudaEventRecord(s->ev_in[b], s->h2d));
+    CU(cudaStreamWaitEvent(st, s->ev_in[b], 0));
+    const int rc = patdnn_stack_run(s, s->p_in[b], s->p_out[b], stream);
+    if (rc) return rc;
+    CU(cudaEventRecord(s->ev_run[b], st));
+    CU(cudaStreamWaitEvent(s->d2h, s->ev_run[b], 0));
+    CU(cudaMemcpyAsync(out_host, s->p_out[b], s->out_bytes, cudaMemcpyDeviceToHost, s->d2h));
+    CU(cudaEventRecord(s->ev_out[b], s->d2h));
+    ++s->submitted;
+    return PATDNN_OK;
+}
+
+int patdnn_stack_wait_host(patdnn_stack s) {
+    if (!s) return PATDNN_E_NULL;
+    if (s->waited >= s->submitted) return PATDNN_OK;
+    CU(cudaEventSynchronize(s->ev_out[s->waited & 1]));
+    ++s->waited;
+    return PATDNN_OK;
+}
+
 int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, int32_t *W) {
     if (!s || !N || !F || !H || !W) return PATDNN_E_NULL;
     *N = s->oN; *F = s->oF; *H = s->oH; *W = s->oW;
@@ -615,6 +659,15 @@ int patdnn_stack_free(patdnn_stack s) {
         if (s->buf[b]) cudaFree(s->buf[b]);
     if (s->d_in) cudaFree(s->d_in);
     if (s->d_out) cudaFree(s->d_out);
+    for (int b = 0; b < 2; ++b) {
+        if (s->p_in[b]) cudaFree(s->p_in[b]);
+        if (s->p_out[b]) cudaFree(s->p_out[b]);
+        if (s->ev_in[b]) cudaEventDestroy(s->ev_in[b]);
+        if (s->ev_run[b]) cudaEventDestroy(s->ev_run[b]);
+        if (s->ev_out[b]) cudaEventDestroy(s->ev_out[b]);
+    }
+    if (s->h2d) cudaStreamDestroy(s->h2d);
+    if (s->d2h) cudaStreamDestroy(s->d2h);
     delete s;
     return PATDNN_OK;
 }

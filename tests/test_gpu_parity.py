@@ -298,3 +298,42 @@ def test_maxpool_matches_oracle():
     B.maxpool2x2(xt, out, 3, 5, 14, 10, B.F32, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert np.array_equal(out.cpu().numpy(), oracle.maxpool2x2(x))
+
+
+def test_pipelined_host_entry_point_matches_the_blocking_one():
+    """submit_host/wait_host over a stream of different batches: every result equals run_host's for that batch, with two
+    batches in flight; a third submission without a wait is refused."""
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, H, W = 2, 20, 24
+    chans = [3, 64, 32]
+    handles = []
+    for i in range(2):
+        L = synth.make_layer(f"p{i}", F=chans[i + 1], C=chans[i], N=N, H=H, W=W, seed=40 + i, prune=0.3 * i, bias_std=0.2,
+                             draw_input=False, w_std=0.3)
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=H, W=W, relu=True, bias=L.bias))
+    stack = B.Stack(handles, [0, 1])
+    rng = np.random.Generator(np.random.PCG64(5))
+    xs = [torch.from_numpy(rng.standard_normal((N, 3, H, W)).astype(np.float32)).pin_memory() for _ in range(5)]
+    ref = []
+    for x in xs:
+        o = np.empty(stack.out_shape(), dtype=np.float32)
+        stack.run_host(x.numpy(), o)
+        ref.append(o)
+    outs = [torch.empty(stack.out_shape(), dtype=torch.float32).pin_memory() for _ in xs]
+    s = torch.cuda.current_stream().cuda_stream
+    stack.submit_host(xs[0].numpy(), outs[0].numpy(), s)
+    stack.submit_host(xs[1].numpy(), outs[1].numpy(), s)
+    with pytest.raises(B.PatdnnError):
+        stack.submit_host(xs[2].numpy(), outs[2].numpy(), s)
+    for i in range(2, 5):
+        stack.wait_host()
+        stack.submit_host(xs[i].numpy(), outs[i].numpy(), s)
+    stack.wait_host()
+    stack.wait_host()
+    stack.wait_host()                                       # nothing outstanding: returns at once
+    for o, r in zip(outs, ref):
+        assert np.array_equal(o.numpy(), r)
+    stack.free()
+    for h in handles:
+        h.free()
