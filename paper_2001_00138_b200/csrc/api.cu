@@ -188,6 +188,7 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
             } else {
                 h->variant = desc->variant;
             }
+            if (desc->N == 0) h->variant = PATDNN_VARIANT_REORDER;   // an empty batch launches nothing: no plan to make
             if (h->variant == PATDNN_VARIANT_TILED && !can_tile) rc = PATDNN_E_SHAPE;
         }
         TiledLayout lay;
@@ -280,10 +281,11 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
 }
 
 int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
-    if (!h || !in || !out) return PATDNN_E_NULL;
+    if (!h) return PATDNN_E_NULL;
     if (!h->on_device) return PATDNN_E_NO_DEVICE;
     const patdnn_desc &d = h->desc;
-    if (d.N == 0) return PATDNN_OK;
+    if (d.N == 0) return PATDNN_OK;                          // an empty batch has no tensors to point at
+    if (!in || !out) return PATDNN_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if (h->variant == PATDNN_VARIANT_DENSE_TC) {

@@ -337,3 +337,51 @@ def test_pipelined_host_entry_point_matches_the_blocking_one():
     stack.free()
     for h in handles:
         h.free()
+
+
+@pytest.mark.parametrize("hw", [(24, 24), (14, 10)])
+def test_fp16_stack_with_pools(hw):
+    """fp16 storage end to end: four layers, two pools; the oracle chain rounds every layer boundary to fp16 like the
+    stored activations (a pool commutes with that rounding)."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, (H, W) = 3, hw
+    chans = [3, 64, 64, 96, 40]
+    pools = [0, 1, 1, 0]
+    x = synth.make_layer("x", F=1, C=3, N=N, H=H, W=W, seed=9, x_dist="normal", dtype="f16").x
+    cur, handles, h, w = x.astype(np.float32), [], H, W
+    for i in range(4):
+        L = synth.make_layer(f"h{i}", F=chans[i + 1], C=chans[i], N=N, H=h, W=w, seed=300 + i, prune=0.0 if i == 0 else 0.5,
+                             bias_std=0.2, draw_input=False, dtype="f16", w_std=float(np.sqrt(2.0 / (4 * chans[i] * 0.6))))
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=h, W=w, dtype=B.F16, relu=True, bias=L.bias))
+        cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+        if pools[i]:
+            cur = oracle.maxpool2x2(cur)
+            h, w = h // 2, w // 2
+        if i < 3:
+            cur = cur.astype(np.float16).astype(np.float32)
+    stack = B.Stack(handles, pools)
+    assert stack.out_shape() == cur.shape
+    out = torch.empty(cur.shape, device="cuda", dtype=torch.float16)
+    stack.run(torch.from_numpy(x).to("cuda", dtype=torch.float16), out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for hd in handles:
+        hd.check()
+    assert_close(out.float().cpu().numpy(), cur, 4 * TOL_F16, f"fp16 stack {hw}")
+    stack.free()
+    for hd in handles:
+        hd.free()
+
+
+def test_empty_batch_is_a_no_op():
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    L = synth.make_layer("z", F=16, C=8, N=1, H=6, W=6, seed=3, draw_input=False)
+    for variant in ("auto", "dense", "tiled", "reorder"):
+        h = B.encode(L.weights, L.mask, L.patterns, N=0, H=6, W=6, relu=True, bias=L.bias, variant=VARIANTS[variant])
+        x = torch.empty((0, 8, 6, 6), device="cuda")
+        y = torch.empty((0, 16, 6, 6), device="cuda")
+        h.conv(x, y, torch.cuda.current_stream().cuda_stream)
+        h.check()
+        h.free()
