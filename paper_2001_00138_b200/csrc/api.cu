@@ -492,7 +492,8 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         patdnn_layer *h = s->layers[i], *nx = s->layers[i + 1];
         const patdnn_desc &d = h->desc;
         if (h->variant == PATDNN_VARIANT_DENSE_TC || s->pool[i] || nx->variant != PATDNN_VARIANT_DENSE_TC || nx->dense.im2col ||
-            nx->dense.Cp != 64 || !smallc_split_supported(d.F, d.C) || std::getenv("PATDNN_NO_SMALLC"))
+            nx->dense.Cp != 64 || !smallc_split_supported(d.F, d.C) || std::getenv("PATDNN_NO_SMALLC") ||
+            static_cast<int64_t>(d.N) * d.C * d.H * d.W >= (int64_t(1) << 31))
             continue;
         s->smallc_w.emplace_back();
         build_smallc_weights(h->fkw, h->bias, s->smallc_w.back());

@@ -38,20 +38,25 @@ conv_smallc_split_kernel(const __grid_constant__ SmallCWeights wt, const T *__re
         const bool ok = pix < P;
         float v[9 * C];
         {
-            const long long q = ok ? pix : 0;
-            const int x = static_cast<int>(q % W);
-            const long long r = q / W;
-            const int y = static_cast<int>(r % H), n = static_cast<int>(r / H);
+            // 32-bit index arithmetic (the launcher checks N*H*W and N*C*H*W < 2^31): 64-bit divisions are subroutines
+            const unsigned q = ok ? static_cast<unsigned>(pix) : 0u;
+            const unsigned uw = static_cast<unsigned>(W), uh = static_cast<unsigned>(H);
+            const unsigned r = q / uw;
+            const int x = static_cast<int>(q - r * uw);
+            const unsigned n = r / uh;
+            const int y = static_cast<int>(r - n * uh);
+            const bool rok[3] = {ok && y >= 1, ok, ok && y + 1 < H};
+            const bool cok[3] = {x >= 1, true, x + 1 < W};
+            const T *base = in + (static_cast<size_t>(n) * C * H + y) * W + x;     // channel 0, centre tap
+            const int plane = H * W;
 #pragma unroll
             for (int c = 0; c < C; ++c)
 #pragma unroll
                 for (int dy = 0; dy < 3; ++dy)
 #pragma unroll
                     for (int dx = 0; dx < 3; ++dx) {
-                        const int yy = y + dy - 1, xx = x + dx - 1;
                         float t = 0.f;
-                        if (ok && yy >= 0 && yy < H && xx >= 0 && xx < W)
-                            t = static_cast<float>(in[((static_cast<size_t>(n) * C + c) * H + yy) * W + xx]);
+                        if (rok[dy] && cok[dx]) t = static_cast<float>(base[c * plane + (dy - 1) * W + (dx - 1)]);
                         v[9 * c + 3 * dy + dx] = t;
                     }
         }
@@ -121,6 +126,7 @@ template <int C>
 cudaError_t launch_c(const SmallCWeights &wt, const void *in, int in_is_half, void *dst, int N, int H, int W, int F, int relu,
                      int Cp, int S, cudaStream_t st) {
     const long long P = static_cast<long long>(N) * H * W;
+    if (P * C >= (1ll << 31)) return cudaErrorInvalidValue;      // the kernel indexes pixels with 32 bits
     const long long blocks_needed = (P + kWarps * 32 - 1) / (kWarps * 32);
     const int grid = static_cast<int>(blocks_needed < 148 * 8 ? blocks_needed : 148 * 8);
     if (in_is_half)
