@@ -33,6 +33,7 @@ ODD_SHAPES = [
     (2, 3, 5, 5, 5, 8, 0.0), (1, 4, 20, 7, 7, 8, 0.3), (3, 8, 33, 14, 14, 12, 0.5), (2, 16, 64, 9, 13, 8, 0.6),
     (1, 5, 7, 1, 1, 4, 0.0), (1, 6, 40, 2, 30, 6, 0.2), (5, 9, 17, 3, 4, 8, 0.4), (2, 20, 130, 16, 16, 8, 0.7),
     (1, 3, 16, 40, 36, 8, 0.0), (4, 12, 24, 6, 10, 12, 0.9), (1, 33, 70, 18, 66, 8, 0.5), (7, 2, 3, 4, 8, 8, 0.0),
+    (1, 1000, 1000, 7, 7, 8, 0.8), (2, 100, 300, 15, 17, 12, 0.6),      # channel counts beyond any tile, not multiples of 64
 ]
 
 
