@@ -651,13 +651,16 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // 3x3 neighbourhood of their pixels straight from the caller's NCHW input, split it, and write the [pixel][k] operand
 // rows (k = 9*c + tap, zero beyond 9*C) into the A ring in the swizzled layout a TMA load would have produced.
 template <int BN, int MT, int TERMS, typename T, bool GATHER>
-__global__ void __launch_bounds__(GATHER ? kHaloThreads + kGatherThreads : kHaloThreads, 1)
+__global__ void __launch_bounds__(GATHER ? kHaloThreads + kGatherThreads : (MT == 2 ? kHaloThreads + 32 : kHaloThreads), 1)
 conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
     constexpr int S = (TERMS == 3) ? 2 : 1;
     constexpr int B_BYTES = BN * 128;
     constexpr bool MERGE = (TERMS == 3) && (BN <= 128);          // see conv_umma_kernel: x_hi * [w_hi | w_lo] in one MMA
     constexpr int ACC_COLS = MERGE ? 2 * BN : BN;
     constexpr int BUF_COLS = MT * ACC_COLS;                      // one accumulator buffer
+    // Double tiles of the TMA-fed kernel have one MMA-issuing thread per accumulator (warp 1 and warp 10): narrow MMAs
+    // cost their issue, not their arithmetic, and two threads issue twice as many.
+    constexpr int ISSUERS = (MT == 2 && !GATHER) ? 2 : 1;
     static_assert(2 * BUF_COLS <= 512, "two accumulator buffers must fit the 512 TMEM columns");
     constexpr int TMEM_COLS = 2 * BUF_COLS < 32 ? 32 : 2 * BUF_COLS;
     extern __shared__ unsigned char smem_raw[];
@@ -684,10 +687,10 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     pdl_trigger();
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
-            mbar_init(bar_fa + 8 * s, GATHER ? kGatherThreads / 32 : 1); mbar_init(bar_ea + 8 * s, 1);
-            mbar_init(bar_fb + 8 * s, 1); mbar_init(bar_eb + 8 * s, 1);
+            mbar_init(bar_fa + 8 * s, GATHER ? kGatherThreads / 32 : 1); mbar_init(bar_ea + 8 * s, ISSUERS);
+            mbar_init(bar_fb + 8 * s, 1); mbar_init(bar_eb + 8 * s, ISSUERS);
         }
-        mbar_init(bar_af, 1); mbar_init(bar_af + 8, 1);
+        mbar_init(bar_af, ISSUERS); mbar_init(bar_af + 8, ISSUERS);
         mbar_init(bar_ae, 8); mbar_init(bar_ae + 8, 8);         // one arrival per epilogue warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -743,7 +746,8 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || (ISSUERS == 2 && warp == kHaloThreads / 32)) {
+        const int mt_lo = (ISSUERS == 2) ? (warp == 1 ? 0 : 1) : 0, mt_hi = (ISSUERS == 2) ? mt_lo + 1 : MT;
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
             constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
@@ -771,6 +775,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                             const uint64_t b_hi = smem_desc_sw128(bbase), b_lo = smem_desc_sw128(bbase + B_BYTES);
 #pragma unroll
                             for (int mt = 0; mt < MT; ++mt) {
+                                if (mt < mt_lo || mt >= mt_hi) continue;                         // the other issuer's tile
                                 const uint32_t arow = abase + (mt * p.TH + r) * row_bytes;       // 1024-byte aligned
                                 const uint64_t a_hi = smem_desc_sw128(arow), a_lo = smem_desc_sw128(arow + a_plane);
                                 const uint32_t acc = tmem_base + buf * BUF_COLS + mt * ACC_COLS;
@@ -992,7 +997,8 @@ cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t 
     }
     DenseParams q = p;
     q.tile_limit = pl.tail_tiles ? pl.n_tiles - pl.tail_tiles : 0;
-    cudaError_t e = launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 1, pl.mapA, pl.mapB, q);
+    cudaError_t e = launch_pdl(kern, dim3(pl.grid), dim3(MT == 2 ? kHaloThreads + 32 : kHaloThreads), pl.smem_bytes, st, 1, pl.mapA,
+                               pl.mapB, q);
     if (e == cudaSuccess && pl.tail_tiles) e = launch_tail<BN, TERMS, T>(pl, p, st, pl.n_tiles - pl.tail_tiles);
     return e;
 }
