@@ -1061,18 +1061,21 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
     const int total_iters = pl.taps * pl.KB;
     // a 2-way split of a 128-wide tile exchanges a quarter of what a 4-way split of a 256-wide tile does (measured faster)
-    while (pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 < 100) pl.BN /= 2;
-    while (pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 4 < 100) pl.BN /= 2;
+    const bool keep_bn = std::getenv("PATDNN_BN_KEEP") != nullptr;   // tuning override: no narrowing
+    while (!keep_bn && pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 < 100) pl.BN /= 2;
+    while (!keep_bn && pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 8 < 60) pl.BN /= 2;   // 8-way split still too few CTAs
     if (force_bn) pl.BN = force_bn;
     pl.poolable = (pool_tiles && best > 0) ? 1 : 0;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
     int ks = 1;
-    // one wave only: with ~200 KB of shared memory per CTA, 148 CTAs fit as clusters of 2, 132 as clusters of 4
-    // (occupancy query); a second wave costs more than the shorter loop saves
+    // one wave only: with ~200 KB of shared memory per CTA, 148 CTAs fit as clusters of 2, 132 as clusters of 4, 120 as
+    // clusters of 8 (occupancy query); a second wave costs more than the shorter loop saves
     if (base_grid < 100)
-        while (ks < 4 && base_grid * ks * 2 <= (ks * 2 == 2 ? 148 : 132) && ks * 2 <= total_iters && pl.BN / (ks * 2) >= 8) ks *= 2;
+        while (ks < 8 && base_grid * ks * 2 <= (ks * 2 == 2 ? 148 : (ks * 2 == 4 ? 132 : 120)) && ks * 2 <= total_iters &&
+               pl.BN / (ks * 2) >= 8)
+            ks *= 2;
     if (const char *ov = std::getenv("PATDNN_KSPLIT")) {
         const int want = atoi(ov);
         if ((want == 1 || want == 2 || want == 4 || want == 8) && want <= total_iters && pl.BN / want >= 8) ks = want;
