@@ -1108,6 +1108,12 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
         if (btw && butil >= util_now - (pl.im2col ? 0.30 : 0.02)) {
             const int th = kTileM / btw;
             int mt = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
+            if (mt == 2) {
+                // a double tile costs ~1/0.65 single tiles (measured); with few rounds the finer granularity can win
+                const long long t1 = static_cast<long long>((W + btw - 1) / btw) * ((H + th - 1) / th) * N * pl.n_ftiles;
+                const long long r1 = (t1 + 147) / 148, r2 = (t1 / 2 + 147) / 148;
+                if (0.65 * static_cast<double>(r1) < static_cast<double>(r2)) mt = 1;
+            }
             if (const char *mv = std::getenv("PATDNN_MT")) mt = (atoi(mv) == 2 && pl.BN == 64) ? 2 : 1;
             const int hr = pl.im2col ? 0 : 2;
             const int a_stage = pl.S * (mt * th + hr) * btw * 128;
