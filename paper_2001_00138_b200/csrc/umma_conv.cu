@@ -488,6 +488,19 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    // The weights do not depend on the previous kernel: the producer thread fetches the weight tiles of the first ring
+    // slots before it waits for that kernel, so they travel (from HBM, when the L2 is cold) while it drains.
+    const int npre = iters < stages ? iters : stages;
+    if (threadIdx.x == 0) {
+        for (int it = 0; it < npre; ++it) {
+            const int cb = (it0 + it) / p.taps, tap = (it0 + it) - cb * p.taps;
+            const uint32_t base = smem_u32(smem + static_cast<size_t>(it) * STAGE_BYTES);
+            mbar_expect_tx(bar_full + 8 * it, S * (p.box_bytes + B_BYTES));
+#pragma unroll
+            for (int sp = 0; sp < S; ++sp)
+                tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * it, cb * kKBlock, f0, tap, sp);
+        }
+    }
     pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
     if (threadIdx.x == 0) PATDNN_STAMP(1);
     bool acc_ready = false;                                     // epilogue thread holding a finished K-range partial
@@ -501,11 +514,11 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 const int cb = (it0 + it) / p.taps, tap = (it0 + it) - cb * p.taps;
                 const int r = p.taps == 9 ? tap / 3 : 1, sx = p.taps == 9 ? tap - 3 * r : 1;
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
-                mbar_expect_tx(bar_full + 8 * s, tx_bytes);
+                if (it >= npre) mbar_expect_tx(bar_full + 8 * s, tx_bytes);   // the first slots were armed with their weights
 #pragma unroll
                 for (int sp = 0; sp < S; ++sp) {
                     tma_load_5d(base + sp * A_BYTES, &mapA, bar_full + 8 * s, cb * kKBlock, x0 + sx - 1, y0 + r - 1, n0, sp);
-                    tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * s, cb * kKBlock, f0, tap, sp);
+                    if (it >= npre) tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * s, cb * kKBlock, f0, tap, sp);
                 }
             }
         }
@@ -702,8 +715,6 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
-    if (threadIdx.x == 0) PATDNN_STAMP(1);
 
     auto decode = [&](int t, int &ft, int &x0, int &y0, int &n) {
         ft = t % p.n_ftiles; t /= p.n_ftiles;
@@ -711,6 +722,8 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         const int tiy = t % p.tiles_y; t /= p.tiles_y;
         n = t; x0 = tix * p.TW; y0 = tiy * (MT * p.TH);
     };
+    pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
+    if (threadIdx.x == 0) PATDNN_STAMP(1);
 
     if (warp == 0) {
         if (lane == 0) {
