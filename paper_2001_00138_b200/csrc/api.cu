@@ -421,7 +421,8 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->channels_per_stage = 64; info->channel_splits = p.ksplit;
         // grid_x: CTAs of the main launch (plus, for the one-tile-per-CTA kernel, the tiles of a K-split tail launch, so
         // that it stays the tile count); grid_y: tiles shared by the persistent CTAs; grid_z: tiles given to a tail launch
-        info->grid_x = p.halo ? p.grid : p.grid + p.tail_tiles; info->grid_y = p.halo ? p.n_tiles : 1;
+        info->grid_x = (p.halo || p.pair) ? p.grid : p.grid + p.tail_tiles;
+        info->grid_y = p.pair ? 2 * p.n_tiles : (p.halo ? p.n_tiles : 1);     // CTA pairs: in single-tile units
         info->grid_z = 1 + p.tail_tiles; info->smem_bytes = p.smem_bytes;
         info->entries = static_cast<int64_t>(p.taps) * p.Fp * p.Cp;
     } else {

@@ -135,6 +135,8 @@ struct DensePlan {
     int n_tiles = 0;                       // halo kernel: tiles shared by the persistent CTAs
     int halo = 0, MT = 1, na = 0;          // halo-sharing kernel: accumulator tiles per CTA, A-ring depth (stages = B ring)
     int ksplit = 1, iters_per_split = 0;   // the (channel block, tap) loop cut into ksplit ranges = CTAs of one cluster
+    int pair = 0;                          // CTA-pair kernel (cta_group::2): tiles of 256 pixels x 256 filters, grid = 2 * clusters
+    CUtensorMap mapB_pair{};               // weight box of one CTA of a pair: 128 of the 256 filters
     int gather = 0;                        // im2col layer on the persistent kernel: operand rows gathered in the kernel
     // Tail of a grid that is not a whole number of 148-CTA rounds: the last tail_tiles tiles run as a second launch of
     // the one-tile-per-CTA kernel with the K loop split tail_ks ways (clusters), instead of costing a whole extra round.

@@ -958,6 +958,245 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     }
 }
 
+// ---- CTA-pair variant of the persistent kernel for 256-filter tiles ----------------------------------------------------
+// Two CTAs of a cluster work on one 256-pixel x 256-filter tile with cta_group::2 MMAs (M = 256): each CTA loads the
+// halo boxes of ITS 128 pixels and only HALF of every weight tile (128 of the 256 filters); the tensor cores of both SMs
+// read the two halves.  Per SM the weight traffic from L2 -- what the single-CTA kernel waits for on these layers --
+// halves.  Protocol (barrier arrays sit at the same shared-memory offsets in both CTAs):
+//   full A / full B   live in the leader (cluster rank 0): two arrivals per phase, one arrive.expect_tx from each CTA's
+//                     producer thread with that CTA's byte count; both CTAs' TMA loads complete on the leader's barrier
+//   empty A / empty B one per CTA, released by the leader's MMA thread with one tcgen05.commit per CTA
+//   accumulator full  one per CTA, same; accumulator empty: in the leader, 16 arrivals (8 epilogue warps x 2 CTAs)
+// The leader's MMA thread issues for both; every CTA drains its own 128 TMEM lanes.  No multicast loads.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap *map, uint32_t cluster_bar, int c0, int c1, int c2,
+                                                 int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap *map, uint32_t cluster_bar, int c0, int c1, int c2,
+                                                 int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8, %9, %10, %11, %12}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u), "r"(0u), "r"(0u),
+          "r"(0u), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
+}
+__host__ __device__ constexpr uint32_t instr_desc_m(int fmt, int n, int m) {
+    return (1u << 4) | (static_cast<uint32_t>(fmt) << 7) | (static_cast<uint32_t>(fmt) << 10) |
+           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+template <int TERMS, typename T>
+__global__ void __launch_bounds__(kHaloThreads, 1)
+conv_umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const DenseParams p) {
+    constexpr int BN = 256, BH = 128;                            // filters per tile, filters whose weights this CTA loads
+    constexpr int S = (TERMS == 3) ? 2 : 1;
+    constexpr int B_BYTES = BH * 128;                            // one weight plane of this CTA's half
+    constexpr int TMEM_COLS = 512;                               // two accumulator buffers of 256 columns
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) uint64_t bars[4 * 8 + 4];
+    __shared__ uint32_t tmem_slot;
+    __shared__ float s_bias[2][BN];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const bool leader = rank == 0;
+    const int NA = p.na, NB = p.stages;
+    const int a_plane = p.box_bytes;                             // (TH+2) * TW * 128 bytes
+    const int a_stage = S * a_plane, b_stage = S * B_BYTES;
+    unsigned char *smem_b = smem + NA * a_stage;
+    const uint32_t bar_fa = smem_u32(&bars[0]), bar_ea = smem_u32(&bars[8]), bar_fb = smem_u32(&bars[16]),
+                   bar_eb = smem_u32(&bars[24]), bar_af = smem_u32(&bars[32]), bar_ae = smem_u32(&bars[34]);
+    // the same barriers seen from the cluster: the leader's full/acc-empty barriers, each CTA's empty/acc-full barriers
+    const uint32_t L_fa = map_to_cta(bar_fa, 0), L_fb = map_to_cta(bar_fb, 0), L_ae = map_to_cta(bar_ae, 0);
+    int *status = p.status;
+    const int row_bytes = p.TW * 128;
+    const int pix_tiles = p.tiles_x * p.tiles_y * p.tiles_n;
+    const int pair_tiles = (pix_tiles + 1) / 2;
+    const int n_pairs = p.tile_limit > 0 ? p.tile_limit : p.n_ftiles * pair_tiles;
+    const int KB = p.KB;
+    const int n_clusters = gridDim.x / 2, cluster_id = blockIdx.x / 2;
+
+    pdl_trigger();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 8; ++s) {
+            mbar_init(bar_fa + 8 * s, 2); mbar_init(bar_ea + 8 * s, 1);
+            mbar_init(bar_fb + 8 * s, 2); mbar_init(bar_eb + 8 * s, 1);
+        }
+        mbar_init(bar_af, 1); mbar_init(bar_af + 8, 1);
+        mbar_init(bar_ae, 16); mbar_init(bar_ae + 8, 16);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                          // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    pdl_wait();
+
+    // pair q: filter tile ft (fastest), pixel tiles 2*pp and 2*pp+1; this CTA takes pixel tile 2*pp + rank
+    auto decode = [&](int q, int &ft, int &x0, int &y0, int &n) {
+        ft = q % p.n_ftiles;
+        int t = 2 * (q / p.n_ftiles) + static_cast<int>(rank);
+        const int tix = t % p.tiles_x; t /= p.tiles_x;
+        const int tiy = t % p.tiles_y; t /= p.tiles_y;
+        n = t; x0 = tix * p.TW; y0 = tiy * p.TH;                 // an odd last tile gives n == N: loads read zeros, nothing is stored
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int ia = 0, ib = 0;
+            bool ok = true;
+            for (int q = cluster_id; q < n_pairs && ok; q += n_clusters) {
+                int ft, x0, y0, n;
+                decode(q, ft, x0, y0, n);
+                const int f0 = ft * BN + static_cast<int>(rank) * BH;
+                for (int cb = 0; cb < KB && ok; ++cb) {
+                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                        const int sa = ia % NA, ua = ia / NA;
+                        if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
+                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                        mbar_expect_tx_cluster(L_fa + 8 * sa, S * a_plane);
+#pragma unroll
+                        for (int sp = 0; sp < S; ++sp)
+                            tma_load_5d_pair(abase + sp * a_plane, &mapA, L_fa + 8 * sa, cb * kKBlock, x0 + sx - 1, y0 - 1, n, sp);
+                        ++ia;
+                        for (int r = 0; r < 3; ++r) {
+                            const int sb = ib % NB, ub = ib / NB;
+                            if (ub > 0 && !mbar_wait(bar_eb + 8 * sb, (ub - 1) & 1, status, 1)) { ok = false; break; }
+                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            mbar_expect_tx_cluster(L_fb + 8 * sb, S * B_BYTES);
+#pragma unroll
+                            for (int sp = 0; sp < S; ++sp)
+                                tma_load_4d_pair(bbase + sp * B_BYTES, &mapB, L_fb + 8 * sb, cb * kKBlock, f0, r * 3 + sx, sp);
+                            ++ib;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = instr_desc_m(TERMS == 3 ? 1 : 0, BN, 256);
+            const uint32_t P_ea = map_to_cta(bar_ea, 1), P_eb = map_to_cta(bar_eb, 1), P_af = map_to_cta(bar_af, 1);
+            int ia = 0, ib = 0, j = 0;
+            bool ok = true;
+            for (int q = cluster_id; q < n_pairs && ok; q += n_clusters, ++j) {
+                const int buf = j & 1, ub2 = j >> 1;
+                if (ub2 > 0 && !mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2)) { ok = false; break; }
+                tc_fence_after();
+                bool first = true;
+                for (int cb = 0; cb < KB && ok; ++cb) {
+                    for (int sx = 0; sx < 3 && ok; ++sx) {
+                        const int sa = ia % NA, ua = ia / NA;
+                        ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
+                        if (!ok) break;
+                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                        for (int r = 0; r < 3 && ok; ++r) {
+                            const int sb = ib % NB, ub = ib / NB;
+                            ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            const uint64_t b_hi = smem_desc_sw128(bbase), b_lo = smem_desc_sw128(bbase + B_BYTES);
+                            const uint32_t arow = abase + r * row_bytes;
+                            const uint64_t a_hi = smem_desc_sw128(arow), a_lo = smem_desc_sw128(arow + a_plane);
+                            const uint32_t acc = tmem_base + buf * BN;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint64_t koff = static_cast<uint64_t>(2 * k);
+                                umma_f16_pair(acc, a_hi + koff, b_hi + koff, idesc, (first && k == 0) ? 0u : 1u);
+                                if constexpr (TERMS == 3) {
+                                    umma_f16_pair(acc, a_hi + koff, b_lo + koff, idesc, 1u);
+                                    umma_f16_pair(acc, a_lo + koff, b_hi + koff, idesc, 1u);
+                                }
+                            }
+                            first = false;
+                            umma_commit_pair(bar_eb + 8 * sb);
+                            umma_commit_pair(P_eb + 8 * sb);
+                            ++ib;
+                        }
+                        if (ok) { umma_commit_pair(bar_ea + 8 * sa); umma_commit_pair(P_ea + 8 * sa); }
+                        ++ia;
+                    }
+                }
+                if (ok) { umma_commit_pair(bar_af + 8 * buf); umma_commit_pair(P_af + 8 * buf); }
+            }
+        }
+    } else {
+        const int q4 = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int m = q4 * 32 + lane;
+        const int ty = m / p.TW, txx = m - ty * p.TW;
+        const int et = threadIdx.x - 64;
+        int j = 0;
+        for (int q = cluster_id; q < n_pairs; q += n_clusters, ++j) {
+            const int buf = j & 1;
+            int ft, x0, y0, n;
+            decode(q, ft, x0, y0, n);
+            const int f0 = ft * BN;
+            for (int i = et; i < BN; i += 256) s_bias[buf][i] = (f0 + i < p.F) ? p.bias[f0 + i] : 0.f;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (!mbar_wait(bar_af + 8 * buf, (j >> 1) & 1, status, 3)) break;
+            tc_fence_after();
+            const int y = y0 + ty, x = x0 + txx;
+            const bool pix_ok = n < p.N && y < p.H && x < p.W;
+#pragma unroll 1
+            for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + buf * BN + c0, v);
+                float a[32];
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) a[jj] = __uint_as_float(v[jj]);
+                emit_chunk<32, T>(p, a, &s_bias[buf][c0], f0 + c0, n, y, x, pix_ok);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(L_ae + 8 * buf);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                          // nobody's shared memory or TMEM goes away under its peer
+    if (warp == 2) {
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1016,7 +1255,23 @@ cudaError_t launch_halo(const DensePlan &pl, const DenseParams &p, cudaStream_t 
     return e;
 }
 
+template <int TERMS, typename T>
+cudaError_t launch_pair(const DensePlan &pl, const DenseParams &p, cudaStream_t st, bool prep) {
+    auto kern = conv_umma_pair_kernel<TERMS, T>;
+    if (prep) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        if (e == cudaSuccess && pl.tail_tiles)
+            e = cudaFuncSetAttribute(conv_umma_kernel<256, TERMS, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        return e;
+    }
+    DenseParams q = p;
+    q.tile_limit = pl.tail_tiles ? pl.n_tiles - pl.tail_tiles : 0;      // in pair tiles
+    return launch_pdl(kern, dim3(pl.grid), dim3(kHaloThreads), pl.smem_bytes, st, 2, pl.mapA, pl.mapB_pair, q);
+}
+
 cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStream_t st, bool prep) {
+    if (pl.pair)
+        return dtype == PATDNN_F16 ? launch_pair<1, __half>(pl, p, st, prep) : launch_pair<3, float>(pl, p, st, prep);
     if (pl.halo) {
 #define PATDNN_HALO(bn, mt)                                                                                        \
     if (pl.BN == bn && pl.MT == mt)                                                                                \
@@ -1150,6 +1405,44 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             }
         }
     }
+    // 256-filter tiles with enough pixel tiles: CTA pairs (cta_group::2), each CTA loading half of every weight tile.
+    // Half-size weight stages also let the 28-pixel-wide halo boxes fit.  Opt-in (PATDNN_PAIR=1): correct, but measured
+    // 8-12 % slower than the single-CTA kernels on the 56x56 and 28x28 layers at batch 32 -- those are not bound by the
+    // weight traffic this halves.
+    const char *pv = std::getenv("PATDNN_PAIR");
+    if (pl.BN == 256 && pl.ksplit == 1 && !pl.im2col && !pool_tiles && pv && pv[0] == '1' && !(hv && hv[0] == '0')) {
+        const double util_free = static_cast<double>(N) * H * W / (static_cast<double>(ptiles) * kTileM);
+        int btw = 0; double butil = 0;
+        for (int tw : {32, 16, 8}) {
+            const int th = kTileM / tw;
+            const double u = static_cast<double>(H) * W /
+                             (static_cast<double>((W + tw - 1) / tw) * tw * static_cast<double>((H + th - 1) / th) * th);
+            const bool fits = 2 * pl.S * (th + 2) * tw * 128 + 2 * pl.S * 128 * 128 <= 218 * 1024;
+            if (fits && u > butil + 1e-9) { butil = u; btw = tw; }
+        }
+        if (btw && butil >= util_free - 0.02) {
+            const int th = kTileM / btw;
+            const int tx = (W + btw - 1) / btw, ty = (H + th - 1) / th;
+            const int pix_tiles = tx * ty * N;
+            const int n_pairs = ((pix_tiles + 1) / 2) * pl.n_ftiles;
+            if (n_pairs >= 74) {
+                const int a_stage = pl.S * (th + 2) * btw * 128, b_stage = pl.S * 128 * 128;
+                int na = 2, nb = 2;
+                const int budget = 218 * 1024;
+                while (nb < 6 && na * a_stage + (nb + 1) * b_stage <= budget) ++nb;
+                while (na < 3 && (na + 1) * a_stage + nb * b_stage <= budget) ++na;
+                pl.pair = 1; pl.halo = 0; pl.MT = 1; pl.gather = 0;
+                pl.TW = btw; pl.TH = th; pl.TN = 1; pl.tiles_x = tx; pl.tiles_y = ty; pl.tiles_n = N;
+                pl.box_bytes = (th + 2) * btw * 128;
+                pl.na = na; pl.stages = nb;
+                pl.smem_bytes = na * a_stage + nb * b_stage + 1024;
+                pl.n_tiles = n_pairs;                            // pair tiles
+                pl.grid = 2 * std::min(n_pairs, 74);
+                pl.tail_tiles = 0;
+                return;
+            }
+        }
+    }
     // Round quantisation: T equal tiles on 148 SMs take ceil(T/148) rounds.  When the last round is nearly empty its
     // tiles go to a second launch whose K loop is split over clusters (largest split that still fits one wave).
     const char *tv = std::getenv("PATDNN_TAIL");
@@ -1211,11 +1504,20 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
         cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)pl.S};
         cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)W * pl.Cp * 2, (cuuint64_t)H * W * pl.Cp * 2,
                                  (cuuint64_t)N * H * W * pl.Cp * 2};
-        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)(pl.halo ? pl.MT * pl.TH + (pl.im2col ? 0 : 2) : pl.TH),
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.TW, (cuuint32_t)(pl.pair ? pl.TH + 2 : (pl.halo ? pl.MT * pl.TH + (pl.im2col ? 0 : 2) : pl.TH)),
                              (cuuint32_t)pl.TN, 1};
         cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (enc(&pl.mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    if (pl.pair) {
+        cuuint64_t dims[4] = {(cuuint64_t)pl.Cp, (cuuint64_t)pl.Fp, (cuuint64_t)pl.taps, (cuuint64_t)pl.S};
+        cuuint64_t strides[3] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)pl.Fp * pl.Cp * 2, (cuuint64_t)pl.taps * pl.Fp * pl.Cp * 2};
+        cuuint32_t box[4] = {(cuuint32_t)kKBlock, 128u, 1, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        if (enc(&pl.mapB_pair, dt, 4, d_w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return PATDNN_E_CUDA;
     }
     if (pl.tail_tiles) {

@@ -1,4 +1,6 @@
 """Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs."""
+import os
+
 import numpy as np
 import pytest
 
@@ -386,3 +388,34 @@ def test_empty_batch_is_a_no_op():
         h.conv(x, y, torch.cuda.current_stream().cuda_stream)
         h.check()
         h.free()
+
+
+@pytest.mark.parametrize("shape", [(20, 96, 256, 56, 56), (37, 64, 300, 28, 28), (41, 128, 512, 16, 16)])
+def test_cta_pair_kernel(shape, monkeypatch):
+    """The opt-in cta_group::2 kernel (two CTAs per 256-pixel x 256-filter tile, each loading half of the weights): same
+    layer as the default kernels, odd pixel-tile counts and padded filter tiles included."""
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    monkeypatch.setenv("PATDNN_PAIR", "1")
+    N, C, F, H, W = shape
+    L = synth.make_layer("pair", F=F, C=C, N=N, H=H, W=W, seed=N + F, prune=0.6, bias_std=0.2, draw_input=False,
+                         w_std=float(np.sqrt(2.0 / (4 * C * 0.4))))
+    rng = np.random.Generator(np.random.PCG64(N))
+    x = rng.random((N, C, H, W), dtype=np.float32)
+    layer = B.encode(L.weights, L.mask, L.patterns, N=N, H=H, W=W, relu=True, bias=L.bias, variant=VARIANTS["dense"])
+    plan = layer.plan()
+    assert plan["grid_x"] == 148 and plan["grid_y"] > 148          # 74 clusters of two CTAs
+    out = torch.full((N, F, H, W), float("nan"), device="cuda")
+    layer.conv(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
+    layer.check()
+    got = out.cpu().numpy()
+    assert np.all(np.isfinite(got))
+    import oracle
+    pts = [(0, 0, 0, 0), (N - 1, F - 1, H - 1, W - 1), (N - 1, 0, H - 1, 0), (0, F - 1, 0, W - 1)]
+    for _ in range(250):
+        pts.append((int(rng.integers(N)), int(rng.integers(F)), int(rng.integers(H)), int(rng.integers(W))))
+    ref = np.asarray([oracle.conv3x3_point(x, L.weights, L.mask, L.bias, True, *pt) for pt in pts])
+    vals = np.asarray([got[pt] for pt in pts])
+    rms = float(np.sqrt(np.mean(got.astype(np.float64) ** 2)))
+    assert np.all(np.abs(vals - ref) <= TOL_F32 * np.maximum(np.abs(ref), rms))
+    layer.free()
