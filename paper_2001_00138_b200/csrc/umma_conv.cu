@@ -22,7 +22,7 @@
 //                in TMEM, and releases the stage with tcgen05.commit;
 //       warps 2-5 epilogue: tcgen05.ld the accumulator, bias + ReLU, store NCHW.
 // Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves through the normal exit
-// (TMEM is always deallocated).  No cluster multicast anywhere.
+// (TMEM is always deallocated).  Every TMA load is issued by, and lands in, one CTA only.
 #include <cuda.h>
 #include <type_traits>
 #include <cuda_bf16.h>
@@ -967,7 +967,7 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
 //                     producer thread with that CTA's byte count; both CTAs' TMA loads complete on the leader's barrier
 //   empty A / empty B one per CTA, released by the leader's MMA thread with one tcgen05.commit per CTA
 //   accumulator full  one per CTA, same; accumulator empty: in the leader, 16 arrivals (8 epilogue warps x 2 CTAs)
-// The leader's MMA thread issues for both; every CTA drains its own 128 TMEM lanes.  No multicast loads.
+// The leader's MMA thread issues for both; every CTA drains its own 128 TMEM lanes.  Each load lands in one CTA only.
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
