@@ -603,6 +603,7 @@ def main():
         "gpu_launches": int(r["launches"]), "graph_ms_per_step": r["graph_ms_per_step"],
         "roofline": {"bound": "tensor", "achieved": tc_ach, "peak": tc_peak, "unit": "TFLOP/s",
                      "frac": tc_ach / tc_peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "frac_of_burst_peak": tc_ach / float(peaks.get("bf16_tflops", tc_peak)),
                      "peak_source": f"{peak_kind} bf16 cuBLAS peak (sustained, kernel timed inside a long step)",
                      "kernel": "conv_umma_halo_kernel / conv_umma_kernel (tcgen05 implicit GEMM, bf16 hi/lo split, three "
                                "products per fp32 product); achieved = executed 16-bit MMA flops / summed launch time of "
