@@ -419,3 +419,73 @@ def test_cta_pair_kernel(shape, monkeypatch):
     rms = float(np.sqrt(np.mean(got.astype(np.float64) ** 2)))
     assert np.all(np.abs(vals - ref) <= TOL_F32 * np.maximum(np.abs(ref), rms))
     layer.free()
+
+
+def _fuzz_cases(n, seed):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    cases = []
+    for _ in range(n):
+        N = int(rng.choice([1, 1, 2, 3, 5, 9, 17, 40]))
+        C = int(rng.choice([1, 2, 3, 4, 7, 8, 16, 31, 64, 65, 100, 130, 200]))
+        F = int(rng.choice([1, 3, 8, 16, 33, 64, 65, 100, 128, 129, 200, 260]))
+        H = int(rng.integers(1, 41))
+        W = int(rng.integers(1, 41))
+        cases.append((N, C, F, H, W, str(rng.choice(["f32", "f16"])), float(rng.choice([0.0, 0.3, 0.7])), bool(rng.integers(2)),
+                      9000 + len(cases)))
+    return cases
+
+
+@pytest.mark.parametrize("case", _fuzz_cases(36, 2024))
+def test_random_layers_all_planner_paths(case):
+    """Seeded random shapes through the planner (AUTO) and the tensor-core variant: whatever kernel, box, split, tail or
+    gather the plan picks, the layer equals the oracle."""
+    N, C, F, H, W, dtype, prune, relu, seed = case
+    if N * F * H * W * C > 3e8:
+        N = 1
+    L = synth.make_layer("fz", F=F, C=C, N=N, H=H, W=W, seed=seed, n_patterns=8, prune=prune, bias_std=0.2,
+                         x_dist="normal", dtype=dtype, relu=relu)
+    ref = oracle_layer(L)
+    tol = TOL_F16 if dtype == "f16" else TOL_F32
+    for variant in ("auto", "dense"):
+        got, _ = gpu_layer(L, variant=VARIANTS[variant])
+        assert_close(got, ref, tol, f"{case}/{variant}")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_stacks(seed):
+    """Seeded random three- and four-layer stacks (channel counts, extents, pools, variants): every hand-over between the
+    kernel families and every fused pool/first-layer path the stack chooses must reproduce the chained oracle."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    rng = np.random.Generator(np.random.PCG64(7000 + seed))
+    nl = int(rng.integers(3, 5))
+    N = int(rng.choice([1, 2, 4, 9]))
+    H, W = int(rng.integers(8, 41)), int(rng.integers(8, 41))
+    chans = [int(rng.choice([1, 3, 4, 16, 40]))] + [int(rng.choice([16, 64, 64, 96, 130])) for _ in range(nl)]
+    pools = [int(rng.integers(2)) for _ in range(nl)]
+    x = rng.standard_normal((N, chans[0], H, W)).astype(np.float32)
+    cur, handles, h, w = x, [], H, W
+    for i in range(nl):
+        if pools[i] and (h < 2 or w < 2):
+            pools[i] = 0
+        L = synth.make_layer(f"rs{i}", F=chans[i + 1], C=chans[i], N=N, H=h, W=w, seed=8000 + 10 * seed + i,
+                             prune=0.0 if i == 0 else 0.5, bias_std=0.2, draw_input=False,
+                             w_std=float(np.sqrt(2.0 / (4 * chans[i] * (1.0 if i == 0 else 0.5)))))
+        variant = VARIANTS[str(rng.choice(["auto", "auto", "dense", "reorder"]))]
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=h, W=w, relu=True, bias=L.bias, variant=variant))
+        cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+        if pools[i]:
+            cur = oracle.maxpool2x2(cur)
+            h, w = h // 2, w // 2
+    stack = B.Stack(handles, pools)
+    assert stack.out_shape() == cur.shape
+    out = torch.empty(cur.shape, device="cuda")
+    stack.run(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for hd in handles:
+        hd.check()
+    assert_close(out.cpu().numpy(), cur, 5 * TOL_F32, f"random stack {seed}: {chans} pools {pools} {H}x{W} N={N}")
+    stack.free()
+    for hd in handles:
+        hd.free()
