@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatdnn.so")
-SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "smallc_split.cu", "tiled_inst_4x8.cu",
+SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "smallc_split.cu", "smallc_jit.cu", "tiled_inst_4x8.cu",
            "tiled_inst_4x4.cu", "tiled_inst_2x8.cu", "fkw_encoder.cpp", "tiled_plan.cpp"]
 HEADERS = ["kernels.hpp", "kernels_tiled.cuh", "fkw_encoder.hpp", os.path.join("generated", "tiled_cases.inc"),
            os.path.join("..", "..", "include", "patdnn.h")]
@@ -58,7 +58,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         if p.returncode:
             raise RuntimeError(f"nvcc failed on {s}")
     tmp = LIB + f".tmp{os.getpid()}"
-    subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])   # cudart static; driver API via entry points
+    subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a", "-ldl"])   # cudart static; driver API via entry points
     os.replace(tmp, LIB)
     return LIB
 

@@ -87,6 +87,7 @@ struct patdnn_stack_s {
     int64_t submitted = 0, waited = 0;
     std::vector<int> smallc;                  // per layer: index into smallc_w, or -1
     std::vector<SmallCWeights> smallc_w;      // few-channel layers fused with the layout of the tensor-core layer after them
+    std::vector<SmallCJit *> smallc_jit;      // the same layers as run-time generated code (nullptr: static kernel)
     void *buf[2] = {nullptr, nullptr};
     void *d_in = nullptr, *d_out = nullptr;   // staging buffers of patdnn_stack_run_host
     size_t buf_bytes = 0, in_bytes = 0, out_bytes = 0;
@@ -498,6 +499,7 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
             continue;
         s->smallc_w.emplace_back();
         build_smallc_weights(h->fkw, h->bias, s->smallc_w.back());
+        s->smallc_jit.push_back(smallc_jit_build(h->fkw, h->bias, d.C, d.relu, d.dtype == PATDNN_F16, nullptr));
         s->smallc[i] = static_cast<int>(s->smallc_w.size()) - 1;
     }
     s->oN = N; s->oF = C; s->oH = H; s->oW = W;
@@ -571,8 +573,10 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
             }
             if (s->smallc[i] >= 0) {
                 patdnn_layer *nx = s->layers[i + 1];
-                cudaError_t e = launch_smallc_split(s->smallc_w[s->smallc[i]], cur, d.dtype == PATDNN_F16, nx->d_act, d.N, d.C, d.H,
-                                                    d.W, d.F, d.relu, nx->dense.Cp, nx->dense.S, st);
+                SmallCJit *jit = s->smallc_jit[s->smallc[i]];
+                cudaError_t e = jit ? smallc_jit_launch(jit, cur, nx->d_act, d.N, d.H, d.W, st)
+                                    : launch_smallc_split(s->smallc_w[s->smallc[i]], cur, d.dtype == PATDNN_F16, nx->d_act, d.N, d.C,
+                                                          d.H, d.W, d.F, d.relu, nx->dense.Cp, nx->dense.S, st);
                 if (e != cudaSuccess) return cuda_fail(e, "few-channel kernel launch");
                 g_launches.fetch_add(1, std::memory_order_relaxed);
                 direct = true;
@@ -670,6 +674,7 @@ int patdnn_stack_free(patdnn_stack s) {
         if (s->ev_run[b]) cudaEventDestroy(s->ev_run[b]);
         if (s->ev_out[b]) cudaEventDestroy(s->ev_out[b]);
     }
+    for (SmallCJit *j : s->smallc_jit) smallc_jit_free(j);
     if (s->h2d) cudaStreamDestroy(s->h2d);
     if (s->d2h) cudaStreamDestroy(s->d2h);
     delete s;

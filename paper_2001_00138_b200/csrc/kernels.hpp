@@ -5,6 +5,7 @@
 
 #include <cstdint>
 #include <cstdlib>
+#include <string>
 #include <vector>
 
 #include "fkw_encoder.hpp"
@@ -176,6 +177,13 @@ void build_smallc_weights(const Fkw &fkw, const std::vector<float> &bias, SmallC
 // in: NCHW (fp32 or fp16); dst: [S][N][H][W][Cp] split operands of the next layer (Cp = 64), bias + ReLU applied.
 cudaError_t launch_smallc_split(const SmallCWeights &wt, const void *in, int in_is_half, void *dst, int N, int C, int H, int W,
                                 int F, int relu, int Cp, int S, cudaStream_t st);
+
+// The same layer as code generated for it and compiled at run time (smallc_jit.cu): only the kept weights, as immediates.
+// smallc_jit_build returns nullptr where NVRTC is not available (the caller keeps the static kernel).
+struct SmallCJit;
+SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log);
+cudaError_t smallc_jit_launch(SmallCJit *j, const void *in, void *dst, int N, int H, int W, cudaStream_t st);
+void smallc_jit_free(SmallCJit *j);
 
 bool dense_supported(int F, int C, int N, int H, int W);
 // pool_tiles: only pixel boxes whose epilogue can max-pool in registers (one image per box, 2/4/8/16 pixels wide, starting

@@ -128,15 +128,19 @@ def test_small_channel_layers_gather_their_operand_in_the_kernel(shape, dtype):
     assert_close(got, oracle_layer(L), TOL_F16 if dtype == "f16" else TOL_F32, f"gather {shape} {dtype}")
 
 
+@pytest.mark.parametrize("generated", [True, False])
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
 @pytest.mark.parametrize("shape", [(3, 3, 64, 13, 9), (2, 1, 40, 32, 32), (1, 4, 64, 7, 50), (5, 2, 17, 6, 6)])
-def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype):
+def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype, generated, monkeypatch):
     """CUDA-core layer with C <= 4 and F <= 64 followed by a tensor-core layer: the stack runs ONE kernel for the first
-    layer that writes the second layer's split operands (no NCHW tensor, no layout kernel), then the GEMM."""
+    layer that writes the second layer's split operands (no NCHW tensor, no layout kernel), then the GEMM.  Both forms of
+    that kernel: the code generated for the layer at run time (kept weights as immediates) and the static one."""
     import oracle
     import torch
     from paper_2001_00138_b200 import binding as B
     N, C, F, H, W = shape
+    if not generated:
+        monkeypatch.setenv("PATDNN_NO_JIT", "1")
     dt = B.F16 if dtype == "f16" else B.F32
     tdt = torch.float16 if dtype == "f16" else torch.float32
     L0 = synth.make_layer("f0", F=F, C=C, N=N, H=H, W=W, seed=77 + C, prune=0.0, bias_std=0.3, x_dist="normal", dtype=dtype)
