@@ -231,7 +231,8 @@ def run_suite(args):
         flops, byts, roof_us, bound = layer_costs(L, hbm)
         plan = h.plan()
         print(json.dumps({"suite": tag, "layer": L.name, "batch": N, "variant": variant,
-                          "kernel": {1: "noopt", 2: "reorder", 3: "tiled", 4: "dense_tc"}[plan["variant"]],
+                          "kernel": "generated_fp32" if plan.get("generated") else
+                                    {1: "noopt", 2: "reorder", 3: "tiled", 4: "dense_tc"}[plan["variant"]],
                           "filter_order": "random" if order is not None else "fkr", "K": L.K,
                           "us": round(us, 2), "gflops_nonzero": round(flops / us / 1e3, 1),
                           "roofline_us": round(roof_us, 2), "bound": bound, "frac": round(roof_us / us, 3),
@@ -302,7 +303,8 @@ def suite_cifar_stack(B, synth, torch, hbm, stream):
         print(json.dumps({"suite": "cifar_vgg16_stack", "batch": N, "us": round(us, 1),
                           "gflops_nonzero": round(flops / us / 1e3, 1), "roofline_us": round(roof, 1),
                           "frac": round(roof / us, 3),
-                          "kernels": "".join({3: "t", 4: "D"}.get(h.plan()["variant"], "g") for h in handles),
+                          "kernels": "".join("j" if h.plan().get("generated") else {3: "t", 4: "D"}.get(h.plan()["variant"], "g")
+                                             for h in handles),
                           "timing": "CUDA-graph replay of the chained stack, working set L2-resident"}), flush=True)
         stack.free()
         for h in handles:
@@ -627,7 +629,8 @@ def main():
                                         "and out); stack_frac_step uses the timed step of the chained stack, pools included",
                                 "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
         "layers": [{"name": n, "us": round(u, 2), "roofline_us": round(c[2], 2), "bound": c[3],
-                    "frac": round(c[2] / u, 3), "kernel": {3: "tiled", 4: "dense_tc"}.get(p["variant"], "generic"),
+                    "frac": round(c[2] / u, 3),
+                    "kernel": "generated_fp32" if p.get("generated") else {3: "tiled", 4: "dense_tc"}.get(p["variant"], "generic"),
                     "tile": f"{p['tile_rows']}x{p['tile_cols']}x{p['filters_per_warp']}f", "grid": p["grid_x"]}
                    for n, u, c, p in zip(r["names"], r["layer_us"], r["costs"], r["plans"])],
     }

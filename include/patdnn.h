@@ -186,6 +186,10 @@ typedef struct {
     int32_t smem_bytes;
     int64_t device_bytes;       /* bytes of the private device layout */
     int64_t entries;            /* kernel entries in the device layout (kept kernels plus padding) */
+    int32_t generated;          /* 1: patdnn_conv runs code generated for this layer at encode time (few input channels
+                                 * under PATDNN_VARIANT_AUTO, run-time compiler present); the fields above then describe
+                                 * the kernel it replaces */
+    int32_t reserved;
 } patdnn_plan_info;
 
 PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);

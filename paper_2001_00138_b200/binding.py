@@ -55,7 +55,8 @@ class _PlanInfo(ctypes.Structure):
                 ("filters_per_warp", ctypes.c_int32), ("warps_per_cta", ctypes.c_int32),
                 ("channels_per_stage", ctypes.c_int32), ("channel_splits", ctypes.c_int32),
                 ("grid_x", ctypes.c_int32), ("grid_y", ctypes.c_int32), ("grid_z", ctypes.c_int32),
-                ("smem_bytes", ctypes.c_int32), ("device_bytes", ctypes.c_int64), ("entries", ctypes.c_int64)]
+                ("smem_bytes", ctypes.c_int32), ("device_bytes", ctypes.c_int64), ("entries", ctypes.c_int64),
+                ("generated", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 _lib = None

@@ -71,6 +71,7 @@ struct patdnn_layer {
     int *d_status = nullptr;
     DensePlan dense_static;                  // same plan with its activation map over the fixed scratch array
     bool dense_static_ready = false;
+    SmallCJit *jit_nchw = nullptr;           // few-channel layer on the FP32 pipes: code generated for it (nullptr: tiled/generic kernel)
     DensePlan dense_pool;                    // plan over the same buffers whose epilogue can max-pool (built by a stack)
     int dense_pool_state = 0;                // 0 = not tried, 1 = ready, -1 = this layer's shape has no such plan
     // staging buffers of patdnn_conv_host
@@ -268,6 +269,12 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                     }
                 }
                 if (!rc) h->on_device = true;
+                // AUTO on a few-channel layer that stays on the FP32 pipes: code generated for this layer (kept weights as
+                // immediates) replaces the tiled kernel where the run-time compiler is available
+                if (!rc && desc->variant == PATDNN_VARIANT_AUTO && h->variant != PATDNN_VARIANT_DENSE_TC && desc->N > 0 &&
+                    smallc_split_supported(k.F, k.C) &&
+                    static_cast<int64_t>(desc->N) * std::max(k.C, k.F) * desc->H * desc->W < (int64_t(1) << 31))
+                    h->jit_nchw = smallc_jit_build(k, h->bias, k.C, desc->relu, desc->dtype == PATDNN_F16, nullptr, 1);
             }
         }
     } catch (const std::bad_alloc &) {
@@ -289,7 +296,9 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
     if (!in || !out) return PATDNN_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if (h->variant == PATDNN_VARIANT_DENSE_TC) {
+    if (h->jit_nchw) {
+        e = smallc_jit_launch(h->jit_nchw, in, out, d.N, d.H, d.W, st);
+    } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         return dense_forward(h, h->dense, in, h->d_act, out, st);
     } else if (h->variant == PATDNN_VARIANT_TILED) {
         TiledParams p{};
@@ -378,6 +387,7 @@ int patdnn_check(patdnn_handle h) {
 int patdnn_free(patdnn_handle h) {
     if (!h) return PATDNN_OK;
     for (void *p : h->owned) cudaFree(p);
+    smallc_jit_free(h->jit_nchw);
     delete h;
     return PATDNN_OK;
 }
@@ -406,6 +416,7 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
     std::memset(info, 0, sizeof(*info));
     info->variant = h->variant;
     info->device_bytes = h->device_bytes;
+    info->generated = h->jit_nchw ? 1 : 0;
     if (h->variant == PATDNN_VARIANT_TILED) {
         const TiledPlan &p = h->plan;
         info->tile_rows = p.cfg.TY; info->tile_cols = kTileCols;

@@ -181,7 +181,9 @@ cudaError_t launch_smallc_split(const SmallCWeights &wt, const void *in, int in_
 // The same layer as code generated for it and compiled at run time (smallc_jit.cu): only the kept weights, as immediates.
 // smallc_jit_build returns nullptr where NVRTC is not available (the caller keeps the static kernel).
 struct SmallCJit;
-SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log);
+// nchw_out = 1: the kernel writes the layer's NCHW output (dst = the caller's tensor) instead of split operands.
+SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log,
+                            int nchw_out = 0);
 cudaError_t smallc_jit_launch(SmallCJit *j, const void *in, void *dst, int N, int H, int W, cudaStream_t st);
 void smallc_jit_free(SmallCJit *j);
 

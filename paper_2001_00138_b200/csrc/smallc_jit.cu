@@ -99,7 +99,8 @@ std::string hexfloat(float v) {
 }
 
 // The CUDA C++ source of the layer's kernel.
-std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int C, bool relu, bool half_in) {
+// nchw_out: write the caller's NCHW tensor (a layer run on its own) instead of the next layer's split operands.
+std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int C, bool relu, bool half_in, bool nchw_out) {
     // kept weights per original filter: (k = 9*c + tap, value)
     std::vector<std::vector<std::pair<int, float>>> taps(64);
     std::vector<float> b(64, 0.f);
@@ -118,14 +119,16 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
     const int S = half_in ? 1 : 2;
     o << "typedef unsigned int u32;\n";
     o << "extern \"C\" __global__ void __launch_bounds__(256, 2) patdnn_first_layer(const "
-      << (half_in ? "unsigned short" : "float") << " *__restrict__ in, unsigned short *__restrict__ dst, int N, int H, int W) {\n";
-    o << "  __shared__ __align__(16) unsigned char stage[8][32 * 128];\n";
+      << (half_in ? "unsigned short" : "float") << " *__restrict__ in, "
+      << (nchw_out && !half_in ? "float" : "unsigned short") << " *__restrict__ dst, int N, int H, int W) {\n";
+    if (!nchw_out) o << "  __shared__ __align__(16) unsigned char stage[8][32 * 128];\n";
     o << "  asm volatile(\"griddepcontrol.launch_dependents;\" ::: \"memory\");\n";
     o << "  asm volatile(\"griddepcontrol.wait;\" ::: \"memory\");\n";
     o << "  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;\n";
     o << "  const unsigned P = (unsigned)N * H * W;\n";
     o << "  const size_t plane_out = (size_t)P * 64;\n";
-    o << "  unsigned char *st = stage[warp];\n";
+    if (!nchw_out) o << "  unsigned char *st = stage[warp];\n";
+    else o << "  (void)warp;\n";
     o << "  for (unsigned p0 = (blockIdx.x * 8 + warp) * 32; p0 < P; p0 += gridDim.x * 8 * 32) {\n";
     o << "    const unsigned pix = p0 + lane; const bool ok = pix < P;\n";
     o << "    const unsigned q = ok ? pix : 0u, r_ = q / (unsigned)W; const int x = (int)(q - r_ * W);\n";
@@ -142,7 +145,8 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
     else
         o << "            t = base[c * plane + (dy - 1) * W + (dx - 1)];\n";
     o << "          }\n          v[9 * c + 3 * dy + dx] = t;\n        }\n";
-    o << "    u32 hi[32]" << (S == 2 ? ", lo[32]" : "") << ";\n";
+    if (!nchw_out) o << "    u32 hi[32]" << (S == 2 ? ", lo[32]" : "") << ";\n";
+    else o << "    const size_t obase = (size_t)n * " << fkw.F << " * plane + (size_t)y * W + x;\n";
     for (int g = 0; g < 8; ++g) {
         o << "    {\n";
         for (int j = 0; j < 8; ++j) o << "      float a" << j << " = " << hexfloat(b[8 * g + j]) << ";\n";
@@ -155,6 +159,19 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
                       << "], a" << j << ");\n";
         if (relu)
             for (int j = 0; j < 8; ++j) o << "      a" << j << " = fmaxf(a" << j << ", 0.f);\n";
+        if (nchw_out) {                                          // a warp stores 32 consecutive pixels of one filter plane
+            for (int j = 0; j < 8; ++j) {
+                const int f = 8 * g + j;
+                if (f >= fkw.F) break;
+                if (half_in)
+                    o << "      if (ok) { unsigned short hv; asm(\"cvt.rn.f16.f32 %0, %1;\" : \"=h\"(hv) : \"f\"(a" << j << ")); dst[obase + (size_t)"
+                      << f << " * plane] = hv; }\n";
+                else
+                    o << "      if (ok) dst[obase + (size_t)" << f << " * plane] = a" << j << ";\n";
+            }
+            o << "    }\n";
+            continue;
+        }
         for (int j = 0; j < 8; j += 2) {
             const int w = (8 * g + j) / 2;
             if (S == 2) {
@@ -169,8 +186,8 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
         }
         o << "    }\n";
     }
-    o << "    const int rows = (int)(P - p0 < 32u ? P - p0 : 32u);\n";
-    for (int sp = 0; sp < S; ++sp) {
+    if (!nchw_out) o << "    const int rows = (int)(P - p0 < 32u ? P - p0 : 32u);\n";
+    for (int sp = 0; sp < (nchw_out ? 0 : S); ++sp) {
         const char *arr = sp == 0 ? "hi" : "lo";
         o << "    __syncwarp();\n#pragma unroll\n    for (int ch = 0; ch < 8; ++ch)\n"
           << "      *reinterpret_cast<uint4 *>(st + lane * 128 + ((ch ^ (lane & 7)) << 4)) = make_uint4(" << arr << "[4 * ch], " << arr
@@ -192,12 +209,13 @@ struct SmallCJit {
     CUfunction fn = nullptr;
 };
 
-SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log) {
+SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log,
+                            int nchw_out) {
     if (std::getenv("PATDNN_NO_JIT")) return nullptr;
     const Nvrtc &rt = nvrtc();
     const Driver &dr = driver();
     if (!rt.ok || !dr.ok) { if (log) *log = "NVRTC or the driver entry points are not available"; return nullptr; }
-    const std::string src = generate_source(fkw, bias, C, relu != 0, is_half != 0);
+    const std::string src = generate_source(fkw, bias, C, relu != 0, is_half != 0, nchw_out != 0);
     nvrtcProgram prog = nullptr;
     if (rt.CreateProgram(&prog, src.c_str(), "patdnn_first_layer.cu", 0, nullptr, nullptr) != 0) return nullptr;
     const char *opts[] = {"--gpu-architecture=sm_100a", "--std=c++17"};

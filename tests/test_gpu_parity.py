@@ -272,6 +272,8 @@ def test_vgg_full_size_sampled(i, N):
         pts.append((int(rng.integers(N)), int(rng.integers(L.F)), int(rng.integers(L.H)), int(rng.integers(L.W))))
     for _ in range(60):     # the last image holds the tiles of a K-split tail launch, where the plan has one
         pts.append((N - 1, int(rng.integers(L.F)), int(rng.integers(L.H)), int(rng.integers(L.W))))
+    if i == 0:
+        assert layer.plan()["generated"] == 1, "the RGB layer under AUTO runs code generated for it"
     if (i, N) in ((5, 32), (8, 32)):
         assert layer.plan()["grid_z"] > 1, "these tile counts are not whole rounds of 148 CTAs: a tail launch is planned"
     ref = np.asarray([oracle.conv3x3_point(x, L.weights, L.mask, L.bias, True, *p) for p in pts])
