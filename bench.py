@@ -600,8 +600,9 @@ def main():
                    "patterns": 8, "connectivity_pruning": "0% layer 1, 60% layers 2-13",
                    "l2": "working set larger than L2 (first activation alone is %d MB); input buffers rotated"
                          % (args.batch * 64 * 224 * 224 * 4 // 2**20) if args.batch >= 8 else "see batch1 leg",
-                   "step": "13 conv layers chained by the library: CUDA-core RGB layer, one layout kernel, 12 tensor-core GEMM "
-                           "kernels writing the next layer's operands directly; the 4 max-pools are taken in epilogues"},
+                   "step": "13 conv layers chained by the library: RGB layer as FP32 code generated for it, 12 tensor-core GEMM "
+                           "layers (some with a K-split tail launch), every kernel writing the next layer's operands directly; "
+                           "the 4 max-pools are taken in epilogues"},
         "clocks": r["clocks"],
         "e2e": {"value": world * r["flops"] / (e2e_ms * 1e-3) / 1e9, "unit": "GFLOP/s",
                 "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "ms_per_step": e2e_ms,
