@@ -7,8 +7,17 @@
  *                            positions of one pattern out of a small fixed set;
  *   connectivity pruning   : whole (filter, channel) kernels are removed.
  * The host side builds the compressed weight storage of Section 5.3 (FKW: offset, reorder, index, stride and
- * weight arrays) after the filter-kernel reorder of Section 5.2 (FKR); the device side runs the branch-free,
- * pattern-specialised, register-reusing loops of Sections 5.2 and 5.4 with a fused bias + ReLU epilogue.
+ * weight arrays) after the filter-kernel reorder of Section 5.2 (FKR).  The device side has several kernels for the
+ * same layer (PATDNN_VARIANT_* below): the paper's scheme on the FP32 pipes -- branch-free, pattern-specialised,
+ * register-reusing loops (Sections 5.2 and 5.4) -- and a dense per-tap reformulation on the tensor cores, which on
+ * this GPU is faster for all but very sparse or very thin layers and is what PATDNN_VARIANT_AUTO normally runs.
+ * Every kernel fuses bias + ReLU.
+ *
+ * The three calls of the paper's problem statement are patdnn_encode, patdnn_conv and patdnn_free, with
+ * patdnn_export / patdnn_decode / patdnn_strerror as inspection helpers.  Everything else declared here
+ * (patdnn_conv_host, patdnn_conv_static, patdnn_check, patdnn_plan, patdnn_stack_*, patdnn_maxpool2x2, the launch
+ * counter, patdnn_debug_wait, and the `variant` and `flags` fields of patdnn_desc) is an addition of this library
+ * with no counterpart in the paper; each says so where it is declared.
  *
  * Conventions used by every call
  *   - tap t = 3*r + s (r = kernel row, s = kernel column); a pattern is a 9-bit mask, bit t set = tap t kept,
@@ -55,8 +64,16 @@ enum {
 
 enum { PATDNN_F32 = 0, PATDNN_F16 = 1 };   /* storage type of weights and activations; accumulation is fp32 */
 
-/* Kernel variants.  AUTO picks the tiled kernel planned for the layer's shape; the others exist for the ablation
- * ladder of Section 6.3 (no optimisation -> +reorder -> +load-redundancy elimination). */
+/* Kernel variants (an addition: the paper generates one code version per layer and tunes it offline).
+ * AUTO compares, at encode time, an estimate of the tensor-core variant's time (the zero-padded dense work of nine
+ * per-tap GEMMs, three bf16 products per fp32 product) with the CUDA-core tiled kernel's rate on the kept weights and
+ * takes the faster: DENSE_TC for every layer with more than 7 input channels that is not extremely sparse -- all but
+ * the first layer of the VGG-16 and ResNet-50 shaped workloads -- and, for layers with at most 4 input channels and 64
+ * filters, FP32 code generated for the layer at run time (kept weights as immediates; the tiled kernel where no
+ * run-time compiler is present).  Other few-channel fp32 layers stay on TILED, or on REORDER when their pattern set
+ * is not among the tiled kernel's twelve built-in patterns.  The explicit values run the kernel they name and exist
+ * for the ablation ladder of Section 6.3 (no optimisation -> +reorder -> +load-redundancy elimination -> tensor
+ * cores). */
 enum {
     PATDNN_VARIANT_AUTO = 0,
     PATDNN_VARIANT_NOOPT = 1,     /* original filter order, per-kernel branch on the pattern, global loads */
@@ -79,8 +96,8 @@ typedef struct {
     int32_t filter_order;    /* 0 = filter reorder of Section 5.2; 1 = caller-supplied order (kernel reorder still applies) */
     const int32_t *order;    /* HOST [F] permutation (position -> original filter) when filter_order == 1, else NULL */
     const float *bias;       /* HOST [F] in original filter numbering, or NULL for zeros */
-    int32_t variant;         /* PATDNN_VARIANT_* */
-    int32_t flags;           /* PATDNN_FLAG_* */
+    int32_t variant;         /* PATDNN_VARIANT_* (addition; 0 = AUTO) */
+    int32_t flags;           /* PATDNN_FLAG_* (addition; 0 = none) */
 } patdnn_desc;
 
 /*
@@ -98,8 +115,15 @@ PATDNN_API int patdnn_encode(const float *weights, const uint8_t *mask, const ui
                   const patdnn_desc *desc, patdnn_handle *out);
 
 /*
- * patdnn_conv -- run the layer (Sections 5.2 and 5.4: pattern-ordered branch-free loops with load-redundancy
- * elimination; bias + ReLU fused) asynchronously on `stream`.
+ * patdnn_conv -- run the layer of Section 2.1 / Section 4.2 (formula at the top of this file) asynchronously on
+ * `stream`, with the kernel the handle was planned for:
+ *   TILED     shared-memory tile + halo staging, pattern-ordered branch-free FMA bodies, register patch reused by the
+ *             four taps of a kernel and by the filters of a warp (Sections 5.2 and 5.4), output scattered through reorder[];
+ *   REORDER / NOOPT  the generic kernels of the ablation ladder (any pattern set);
+ *   DENSE_TC  one layout kernel (NCHW -> channels-innermost, operands split into bf16 hi + lo for fp32 layers) into a
+ *             handle-owned scratch buffer, then the tcgen05 implicit GEMM over nine shifted TMA boxes (one launch, plus a
+ *             second launch for the last partial round of tiles where the plan has one);
+ *   generated FP32 code (AUTO, few-channel layers): one kernel.
  *   in   DEVICE [N][C][H][W] of the handle's dtype (float or IEEE half), 16-byte aligned
  *   out  DEVICE [N][F][H][W] of the same dtype, 16-byte aligned; must not overlap `in`
  *   stream  a cudaStream_t (NULL = default stream).  No synchronisation happens inside.
@@ -108,7 +132,7 @@ PATDNN_API int patdnn_encode(const float *weights, const uint8_t *mask, const ui
 PATDNN_API int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream);
 
 /*
- * patdnn_conv_host -- the same operation with HOST buffers: copies `in` to a handle-owned device buffer, runs the
+ * patdnn_conv_host (addition, used by end-to-end measurements) -- the same operation with HOST buffers: copies `in` to a handle-owned device buffer, runs the
  * layer, copies the result back, all on `stream`, and waits for the stream before returning.  Pinned host memory
  * makes the copies asynchronous with respect to other streams.  The device buffers are allocated on first use and
  * live until patdnn_free.
@@ -130,7 +154,8 @@ PATDNN_API int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_
  *     forwarded to patdnn_conv.
  *   - the first call on a device (and the first call for a handle) does set-up work on the host: it looks up the
  *     device address of the array and encodes a tensor map over it.  Make that first call before starting any stream
- *     capture.
+ *     capture.  The call must be made with the device current on which the handle was encoded (PATDNN_E_CUDA
+ *     otherwise); the set-up is serialised between host threads.
  *   - all calls, from every handle, share the one array, which keeps whatever the last call left in it; the kernels
  *     overwrite everything they read, so nothing needs clearing, but two calls that can overlap on the GPU (different
  *     streams without an ordering between them) race on the array and must be serialised by the caller.
@@ -138,7 +163,7 @@ PATDNN_API int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_
 PATDNN_API int patdnn_conv_static(patdnn_handle h, const void *in, void *out, void *stream);
 
 /*
- * patdnn_check -- wait for the device and report whether any kernel launched for this handle gave up on a bounded
+ * patdnn_check (addition) -- wait for the device and report whether any kernel launched for this handle gave up on a bounded
  * device-side wait (PATDNN_E_DEVICE_TIMEOUT) or a CUDA error is pending (PATDNN_E_CUDA).  Synchronous.
  */
 PATDNN_API int patdnn_check(patdnn_handle h);
@@ -171,7 +196,7 @@ PATDNN_API int patdnn_export(patdnn_handle h, patdnn_fkw_view *v);
  * bit for F32 handles and the half-rounded values for F16 handles. */
 PATDNN_API int patdnn_decode(patdnn_handle h, float *dense_out);
 
-/* Planned launch geometry of a handle, for reports and tests. */
+/* Planned launch geometry of a handle, for reports and tests (addition). */
 typedef struct {
     int32_t variant;            /* resolved PATDNN_VARIANT_* */
     int32_t tile_rows, tile_cols;   /* output pixels per thread (rows x columns) */
@@ -182,7 +207,7 @@ typedef struct {
     int32_t grid_x, grid_y, grid_z; /* CUDA-core kernels: the launch grid.  Tensor-core path: grid_x = CTAs of the main
                                      * launch (= tiles for the one-tile-per-CTA kernel), grid_y = tiles shared by the
                                      * persistent CTAs (1 otherwise), grid_z = 1 + tiles handed to a second, K-split
-                                     * launch when the tile count is not a whole number of 148-CTA rounds */
+                                     * launch when the tile count is not a whole number of rounds of one CTA per SM */
     int32_t smem_bytes;
     int64_t device_bytes;       /* bytes of the private device layout */
     int64_t entries;            /* kernel entries in the device layout (kept kernels plus padding) */
@@ -195,6 +220,7 @@ typedef struct {
 PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
 
 /*
+ * Stacks (addition; the paper's framework fuses and chains layers in its graph optimiser, which is out of scope here).
  * A stack chains layers on the device: layer i's output is layer i+1's input, optionally through a 2x2/stride-2
  * max-pool (the VGG-16 arrangement).  The stack owns two ping-pong activation buffers; the handles stay owned by
  * the caller and must outlive the stack.  Between two tensor-core layers no NCHW tensor is formed: the first one's
@@ -229,9 +255,20 @@ PATDNN_API int patdnn_stack_free(patdnn_stack s);
 PATDNN_API int patdnn_maxpool2x2(const void *in, void *out, int32_t N, int32_t C, int32_t H, int32_t W, int32_t dtype,
                       void *stream);
 
-/* Number of this library's kernels launched on the calling thread's behalf since the last reset (for reports). */
+/* Number of this library's kernels launched by the process since the last reset (addition, for reports). */
 PATDNN_API int64_t patdnn_launch_count(void);
 PATDNN_API void patdnn_reset_launch_count(void);
+
+/*
+ * patdnn_debug_wait (addition; test hook of the failure-detection path) -- every device-side wait of the tensor-core
+ * kernels is bounded: after `polls` unsuccessful polls of a barrier (0 = the default, about two seconds) a kernel
+ * records a status word, lets all its roles fall through to the common exit, frees its tensor memory and returns;
+ * patdnn_check then reports PATDNN_E_DEVICE_TIMEOUT and clears the word.  `skip_load_iteration` > 0 makes the
+ * producer of the one-tile-per-CTA kernel leave out the loads of that (1-based) iteration of its channel/tap loop, so
+ * that a test can watch a wait run out; 0 restores normal operation.  Applies to later launches of this handle.
+ * Errors: E_NULL, E_SHAPE (negative iteration).
+ */
+PATDNN_API int patdnn_debug_wait(patdnn_handle h, uint32_t polls, int32_t skip_load_iteration);
 
 PATDNN_API const char *patdnn_strerror(int status);
 PATDNN_API const char *patdnn_last_cuda_error(void);   /* text of the last CUDA failure seen by this thread ("" if none) */

@@ -226,8 +226,18 @@ def check_layer_constraints(weights: np.ndarray, mask: np.ndarray, patterns: Seq
     return kept
 
 
-def storage_bytes(F: int, C: int, K: int, P: int, weight_bytes: int = 4, index_bytes: int = 4) -> Dict[str, int]:
-    """Bytes of the FKW arrays versus a CSR matrix over the same 4K non-zeros (Section 6.4's comparison)."""
-    fkw_index = (F + 1) * index_bytes + F * index_bytes + K * index_bytes + F * (P + 1) * index_bytes
-    csr_index = (F + 1) * index_bytes + 4 * K * index_bytes          # row pointers + one column index per weight
+def storage_bytes(F: int, C: int, K: int, P: int, weight_bytes: int = 4, index_bytes: int = 4,
+                  filter_bytes: int = None, csr_index_bytes: int = None) -> Dict[str, int]:
+    """Bytes of the FKW arrays versus a CSR matrix over the same 4K non-zeros (Section 6.4's comparison).
+
+    ``index_bytes`` is the width of one ``index[]`` entry (one per kept kernel), ``filter_bytes`` the width of the
+    per-filter entries (offset, reorder, stride; default: the same), ``csr_index_bytes`` the width of CSR's column
+    indices and row pointers (default: the same).  The paper's figures (93.4 % of the index bytes and 46.7 % of the
+    total saved at 18x) are matched by about one byte of index per kernel against four bytes per weight in CSR:
+    1 - 1/16 = 93.75 % and 1 - 17/32 = 46.9 % in the limit of long filters.
+    """
+    fb = index_bytes if filter_bytes is None else filter_bytes
+    cb = index_bytes if csr_index_bytes is None else csr_index_bytes
+    fkw_index = (F + 1) * fb + F * fb + K * index_bytes + F * (P + 1) * fb
+    csr_index = (F + 1) * cb + 4 * K * cb                            # row pointers + one column index per weight
     return {"fkw_index": fkw_index, "csr_index": csr_index, "weights": 4 * K * weight_bytes}

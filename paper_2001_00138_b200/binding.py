@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "patdnn_encode", "patdnn_conv", "patdnn_conv_static", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
     "patdnn_stack_free", "patdnn_stack_submit_host", "patdnn_stack_wait_host", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
-    "patdnn_last_cuda_error", "patdnn_version",
+    "patdnn_last_cuda_error", "patdnn_version", "patdnn_debug_wait",
 )
 
 
@@ -79,6 +79,7 @@ def load() -> ctypes.CDLL:
     lib.patdnn_conv_static.argtypes = [vp, vp, vp, vp]
     lib.patdnn_free.argtypes = [vp]
     lib.patdnn_check.argtypes = [vp]
+    lib.patdnn_debug_wait.argtypes = [vp, ctypes.c_uint32, i32]
     lib.patdnn_export.argtypes = [vp, ctypes.POINTER(_FkwView)]
     lib.patdnn_decode.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.patdnn_plan.argtypes = [vp, ctypes.POINTER(_PlanInfo)]
@@ -143,6 +144,11 @@ class Layer:
     def check(self) -> None:
         """patdnn_check: synchronise and raise if a device-side bounded wait expired."""
         _check(load().patdnn_check(self._h), "patdnn_check")
+
+    def debug_wait(self, polls: int, skip_load_iteration: int = 0) -> None:
+        """patdnn_debug_wait: bound of the device-side waits (polls; 0 = default) and the test hook that withholds one
+        iteration's loads so that a wait runs out."""
+        _check(load().patdnn_debug_wait(self._h, polls, skip_load_iteration), "patdnn_debug_wait")
 
     def export(self) -> Dict[str, np.ndarray]:
         v = _FkwView()

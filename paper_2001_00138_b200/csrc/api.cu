@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -20,6 +21,7 @@ namespace {
 
 thread_local std::string g_cuda_error;
 std::atomic<int64_t> g_launches{0};
+std::mutex g_static_mutex;                    // serialises the host-side set-up of patdnn_conv_static
 
 int cuda_fail(cudaError_t e, const char *what) {
     g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -70,7 +72,9 @@ struct patdnn_layer {
     void *d_act = nullptr;
     int *d_status = nullptr;
     DensePlan dense_static;                  // same plan with its activation map over the fixed scratch array
-    bool dense_static_ready = false;
+    bool dense_static_ready = false;         // guarded by g_static_mutex
+    uint32_t spin_limit = 0;                 // patdnn_debug_wait: polls per bounded device-side wait (0 = default)
+    int test_skip_load = 0;                  // patdnn_debug_wait: see DenseParams::test_skip_load
     SmallCJit *jit_nchw = nullptr;           // few-channel layer on the FP32 pipes: code generated for it (nullptr: tiled/generic kernel)
     DensePlan dense_pool;                    // plan over the same buffers whose epilogue can max-pool (built by a stack)
     int dense_pool_state = 0;                // 0 = not tried, 1 = ready, -1 = this layer's shape has no such plan
@@ -105,6 +109,7 @@ static DenseParams dense_params(const patdnn_layer *h, const DensePlan &pl) {
     p.TW = pl.TW; p.TH = pl.TH; p.TN = pl.TN; p.tiles_x = pl.tiles_x; p.tiles_y = pl.tiles_y; p.tiles_n = pl.tiles_n;
     p.n_ftiles = pl.n_ftiles; p.KB = pl.KB; p.stages = pl.stages; p.box_bytes = pl.box_bytes; p.relu = d.relu;
     p.iters_per_split = pl.iters_per_split; p.ksplit = pl.ksplit; p.na = pl.na; p.taps = pl.taps;
+    p.spin_limit = h->spin_limit; p.test_skip_load = h->test_skip_load;
     return p;
 }
 
@@ -121,9 +126,6 @@ static int dense_gemm(patdnn_layer *h, const DensePlan &pl, void *out, const pat
     } else {
         p.mode = 0; p.out = out;
     }
-#ifdef PATDNN_TRACE
-    if (std::getenv("PATDNN_NOSTORE")) p.mode = 9;
-#endif
     cudaError_t e = launch_dense_gemm(pl, p, h->desc.dtype, st);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core kernel launch");
     g_launches.fetch_add(pl.tail_tiles ? 2 : 1, std::memory_order_relaxed);
@@ -185,7 +187,10 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                     const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / tiled_rate + 1.5e-5;
                     // layers with 9*C <= 64 (gathered-neighbourhood GEMM) are store-bound there: measured slower than the
                     // CUDA-core kernel on the RGB first layer, so AUTO leaves them on it unless it cannot run the layer
-                    if (t_dense < t_tiled && (!dp.im2col || !can_tile)) h->variant = PATDNN_VARIANT_DENSE_TC;
+                    // (when the tiled kernel cannot take such a layer -- a pattern outside its builtin table -- fp32 layers
+                    // go to the generic FKW kernel, which is exact to fp32: with so few terms per output the hi/lo split's
+                    // per-product error is not averaged down)
+                    if (t_dense < t_tiled && (!dp.im2col || (!can_tile && desc->dtype == PATDNN_F16))) h->variant = PATDNN_VARIANT_DENSE_TC;
                 }
             } else {
                 h->variant = desc->variant;
@@ -326,24 +331,47 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
 }
 
 int patdnn_conv_static(patdnn_handle h, const void *in, void *out, void *stream) {
-    if (!h || !in || !out) return PATDNN_E_NULL;
+    if (!h) return PATDNN_E_NULL;
     if (!h->on_device) return PATDNN_E_NO_DEVICE;
-    if (h->variant != PATDNN_VARIANT_DENSE_TC) return patdnn_conv(h, in, out, stream);   // no scratch on those paths
     const patdnn_desc &d = h->desc;
-    if (d.N == 0) return PATDNN_OK;
+    if (d.N == 0) return PATDNN_OK;                          // as patdnn_conv: an empty batch has no tensors to point at
+    if (!in || !out) return PATDNN_E_NULL;
+    if (h->variant != PATDNN_VARIANT_DENSE_TC) return patdnn_conv(h, in, out, stream);   // no scratch on those paths
     if (h->dense.gather) return dense_forward(h, h->dense, in, nullptr, out, static_cast<cudaStream_t>(stream));   // no scratch
     const size_t need = static_cast<size_t>(h->dense.S) * d.N * d.H * d.W * h->dense.Cp * 2;
     if (need > kStaticScratchBytes) return PATDNN_E_SCRATCH;
+    // The array lives once per device and its address is baked into the handle's tensor map: the call must run on
+    // the device the handle was encoded on.
+    int dev = -1;
+    CU(cudaGetDevice(&dev));
+    if (dev != h->device) {
+        g_cuda_error = "patdnn_conv_static: the current device is not the device the handle was encoded on";
+        return PATDNN_E_CUDA;
+    }
     void *scratch = nullptr;
-    int rc = static_scratch_address(&scratch);            // first call on this device: cudaGetSymbolAddress
-    if (rc) return cuda_fail(cudaGetLastError(), "cudaGetSymbolAddress(static scratch)");
-    if (!h->dense_static_ready) {                         // first call for this handle: tensor map over the array
-        h->dense_static = h->dense;
-        rc = make_dense_maps(h->dense_static, scratch, h->d_wdense, d.N, d.H, d.W, d.dtype);
-        if (rc) return rc;
-        h->dense_static_ready = true;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        const cudaError_t e = static_scratch_address(&scratch);   // first call on this device: cudaGetSymbolAddress
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+        if (!h->dense_static_ready) {                         // first call for this handle: tensor map over the array
+            h->dense_static = h->dense;
+            const int rc = make_dense_maps(h->dense_static, scratch, h->d_wdense, d.N, d.H, d.W, d.dtype);
+            if (rc) {
+                if (rc == PATDNN_E_CUDA) g_cuda_error = "cuTensorMapEncodeTiled failed";
+                return rc;
+            }
+            h->dense_static_ready = true;
+        }
     }
     return dense_forward(h, h->dense_static, in, scratch, out, static_cast<cudaStream_t>(stream));
+}
+
+int patdnn_debug_wait(patdnn_handle h, uint32_t polls, int32_t skip_load_iteration) {
+    if (!h) return PATDNN_E_NULL;
+    if (skip_load_iteration < 0) return PATDNN_E_SHAPE;
+    h->spin_limit = polls;
+    h->test_skip_load = skip_load_iteration;
+    return PATDNN_OK;
 }
 
 int patdnn_conv_host(patdnn_handle h, const void *in_host, void *out_host, void *stream) {
@@ -505,7 +533,7 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         patdnn_layer *h = s->layers[i], *nx = s->layers[i + 1];
         const patdnn_desc &d = h->desc;
         if (h->variant == PATDNN_VARIANT_DENSE_TC || s->pool[i] || nx->variant != PATDNN_VARIANT_DENSE_TC || nx->dense.im2col ||
-            nx->dense.Cp != 64 || !smallc_split_supported(d.F, d.C) || std::getenv("PATDNN_NO_SMALLC") ||
+            nx->dense.Cp != 64 || !smallc_split_supported(d.F, d.C) || debug_option("smallc", 1) == 0 ||
             static_cast<int64_t>(d.N) * d.C * d.H * d.W >= (int64_t(1) << 31))
             continue;
         s->smallc_w.emplace_back();

@@ -23,6 +23,19 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 #endif
 bool pdl_enabled();
 
+// ---- debugging / tuning overrides and device facts ----------------------------------------------------------------
+// ONE environment variable steers every override: PATDNN_DEBUG="key=value,key=value,...".  Keys (all optional):
+//   pdl=0      launch without programmatic dependent launch        jit=0     no run-time generated first-layer kernel
+//   smallc=0   no fused few-channel first layer in stacks          tile=TYxFR blocking of the CUDA-core tiled kernel
+//   bn=N       cap of the tensor-core filter tile                  bn_keep=1 no narrowing of the filter tile
+//   ksplit=N   cluster split of the channel loop (1, 2, 4, 8)      halo=0    no persistent halo-sharing kernel
+//   mt=N       accumulator tiles per persistent CTA                pair=1    CTA-pair (cta_group::2) kernel
+//   tail=0     no K-split tail launch
+// debug_option returns the integer after "key=", or dflt when the key (or the variable) is absent.
+int debug_option(const char *key, int dflt);
+bool debug_option_text(const char *key, char *buf, size_t cap);   // raw text after "key=" (false when absent)
+int sm_count();                                                   // multiprocessors of the current device (148 if unknown)
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster, Args... args) {
     cudaLaunchConfig_t cfg = {};
@@ -161,10 +174,13 @@ struct DenseParams {
     int tile_base;              // one-tile-per-CTA kernel: index of the first tile this launch covers
     int tile_limit;             // persistent kernel: tiles [0, tile_limit) only (0 = all)
     const void *gather_src;     // gather plans: the layer's NCHW input (fp32 or fp16 as the layer's dtype)
+    uint32_t spin_limit;        // polls a bounded device-side wait may take before it gives up (0 = the default, ~2 s)
+    int test_skip_load;         // test hook of the one-tile-per-CTA kernel: the producer leaves out the loads of its
+                                // (1-based) iteration test_skip_load, so that a bounded wait runs out (0 = off)
 };
 
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // fixed device array behind patdnn_conv_static
-int static_scratch_address(void **ptr);                    // PATDNN_* status; first call per device looks the address up
+cudaError_t static_scratch_address(void **ptr);            // first call per device looks the address up; not thread-safe
 
 // ---- first-layer kernel writing a tensor-core layer's operands (smallc_split.cu) ----------------------------------
 constexpr int kSmallCTaps = 36;            // 9 taps x at most 4 input channels

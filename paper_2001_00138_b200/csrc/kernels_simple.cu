@@ -10,7 +10,10 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
+#include <cstdlib>
+#include <cstring>
 
 #include "kernels.hpp"
 
@@ -116,9 +119,44 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const T *in, T *out, in
     }
 }
 
+bool debug_option_text(const char *key, char *buf, size_t cap) {
+    const char *env = std::getenv("PATDNN_DEBUG");
+    if (!env || !key || cap == 0) return false;
+    const size_t klen = std::strlen(key);
+    for (const char *q = env; *q;) {
+        const char *end = std::strchr(q, ',');
+        const size_t len = end ? static_cast<size_t>(end - q) : std::strlen(q);
+        if (len > klen && std::strncmp(q, key, klen) == 0 && q[klen] == '=') {
+            const size_t n = std::min(len - klen - 1, cap - 1);
+            std::memcpy(buf, q + klen + 1, n);
+            buf[n] = 0;
+            return true;
+        }
+        q += len + (end ? 1 : 0);
+    }
+    return false;
+}
+
+int debug_option(const char *key, int dflt) {
+    char buf[32];
+    return debug_option_text(key, buf, sizeof buf) ? std::atoi(buf) : dflt;
+}
+
 bool pdl_enabled() {
-    static const bool on = [] { const char *v = std::getenv("PATDNN_PDL"); return !(v && v[0] == '0'); }();
+    static const bool on = debug_option("pdl", 1) != 0;
     return on;
+}
+
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); n = 148; }
+        cached[dev] = n;
+    }
+    return cached[dev];
 }
 
 cudaError_t launch_simple(const SimpleParams &p, int variant, int dtype, cudaStream_t stream) {
@@ -137,7 +175,7 @@ cudaError_t launch_simple(const SimpleParams &p, int variant, int dtype, cudaStr
 cudaError_t launch_maxpool2x2(const void *in, void *out, int N, int C, int H, int W, int dtype, cudaStream_t stream) {
     const size_t total = static_cast<size_t>(N) * C * (H / 2) * (W / 2);
     if (total == 0) return cudaSuccess;
-    const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 16));
+    const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, sm_count() * 16));
     if (dtype == 1)
         return launch_pdl(maxpool2x2_kernel<__half>, dim3(blocks), dim3(256), 0, stream, 1, static_cast<const __half *>(in),
                           static_cast<__half *>(out), N * C, H, W);

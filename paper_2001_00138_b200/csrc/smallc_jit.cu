@@ -211,7 +211,7 @@ struct SmallCJit {
 
 SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log,
                             int nchw_out) {
-    if (std::getenv("PATDNN_NO_JIT")) return nullptr;
+    if (debug_option("jit", 1) == 0) return nullptr;
     const Nvrtc &rt = nvrtc();
     const Driver &dr = driver();
     if (!rt.ok || !dr.ok) { if (log) *log = "NVRTC or the driver entry points are not available"; return nullptr; }
@@ -253,7 +253,7 @@ cudaError_t smallc_jit_launch(SmallCJit *j, const void *in, void *dst, int N, in
     const long long P = static_cast<long long>(N) * H * W;
     if (P == 0) return cudaSuccess;
     const long long blocks_needed = (P + 255) / 256;
-    const unsigned grid = static_cast<unsigned>(blocks_needed < 148 * 8 ? blocks_needed : 148 * 8);
+    const unsigned grid = static_cast<unsigned>(blocks_needed < sm_count() * 8 ? blocks_needed : sm_count() * 8);
     CUlaunchConfig cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDimX = grid; cfg.gridDimY = 1; cfg.gridDimZ = 1;

@@ -128,7 +128,7 @@ cudaError_t launch_c(const SmallCWeights &wt, const void *in, int in_is_half, vo
     const long long P = static_cast<long long>(N) * H * W;
     if (P * C >= (1ll << 31)) return cudaErrorInvalidValue;      // the kernel indexes pixels with 32 bits
     const long long blocks_needed = (P + kWarps * 32 - 1) / (kWarps * 32);
-    const int grid = static_cast<int>(blocks_needed < 148 * 8 ? blocks_needed : 148 * 8);
+    const int grid = static_cast<int>(blocks_needed < sm_count() * 8 ? blocks_needed : sm_count() * 8);
     if (in_is_half)
         return launch_pdl(conv_smallc_split_kernel<C, __half>, dim3(grid), dim3(kWarps * 32), 0, st, 1, wt,
                           static_cast<const __half *>(in), static_cast<uint16_t *>(dst), N, H, W, F, relu, Cp, S);

@@ -137,7 +137,8 @@ int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, 
     TiledConfig cfg{};
     int ty = 4, fr = 4;
     if (H < 4 || (H % 4 != 0 && H < 16)) { ty = 2; fr = 8; }
-    if (const char *ov = std::getenv("PATDNN_TILE")) {        // "TYxFR", e.g. 4x4
+    char ov[16];
+    if (debug_option_text("tile", ov, sizeof ov)) {            // "TYxFR", e.g. 4x4
         int a = 0, b = 0;
         if (std::sscanf(ov, "%dx%d", &a, &b) == 2 &&
             ((a == 4 && b == 8) || (a == 4 && b == 4) || (a == 2 && b == 8))) {

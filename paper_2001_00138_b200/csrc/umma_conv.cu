@@ -39,22 +39,6 @@
 
 namespace patdnn {
 
-#ifdef PATDNN_TRACE
-// Debug-only CTA timeline (build with -DPATDNN_TRACE): up to 16 time stamps per CTA, read back by patdnn_trace_read().
-__device__ unsigned long long g_trace[1 << 16];
-__device__ __forceinline__ void trace_stamp(int slot) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (blockIdx.x < (1 << 12)) g_trace[blockIdx.x * 16 + slot] = t;
-}
-#define PATDNN_STAMP(slot) trace_stamp(slot)
-#define PATDNN_TIMED(acc, expr) [&] { const long long t__ = clock64(); const bool r__ = (expr); (acc) += clock64() - t__; return r__; }()
-#define PATDNN_PUT(slot, v) do { if (blockIdx.x < (1 << 12)) g_trace[blockIdx.x * 16 + (slot)] = (unsigned long long)(v); } while (0)
-#else
-#define PATDNN_TIMED(acc, expr) (expr)
-#define PATDNN_PUT(slot, v)
-#define PATDNN_STAMP(slot)
-#endif
 
 namespace {
 
@@ -63,7 +47,13 @@ constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA
 constexpr int kGatherThreads = 256;          // plus eight gather warps for layers whose operand rows are built in the kernel
 constexpr int kTileM = 128;
 constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
-constexpr uint32_t kSpinLimit = 1u << 21;    // bounded mbarrier polling: each poll may block up to ~1 us (hint below)
+constexpr uint32_t kSpinLimit = 1u << 21;    // default bound of mbarrier polling: each poll may block up to ~1 us (hint below)
+
+// Where a bounded wait reports to and how many polls it may take (DenseParams::spin_limit, 0 = the default).
+struct WaitCtx {
+    int *word;
+    uint32_t limit;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -74,8 +64,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Bounded wait: returns false (and leaves *status set) when the phase did not complete within the polling budget.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *status, int code) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &status, int code) {
+    for (uint32_t i = 0; i < status.limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred P1;\n\t"
@@ -84,9 +74,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *st
             : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
         // another role already gave up?  (a global read: only now and then, it would otherwise sit on every wake-up path)
-        if ((i & 15u) == 15u && *reinterpret_cast<volatile int *>(status) != 0) return false;
+        if ((i & 15u) == 15u && *reinterpret_cast<volatile int *>(status.word) != 0) return false;
     }
-    atomicCAS(status, 0, code);
+    atomicCAS(status.word, 0, code);
     return false;
 }
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
@@ -377,9 +367,6 @@ __device__ __forceinline__ void emit_chunk(const DenseParams &p, float (&a)[CNT]
         pix_ok = pix_ok && !(x & 1) && !(y & 1) && x + 1 < p.W && y + 1 < p.H;
     }
     if (!pix_ok) return;
-#ifdef PATDNN_TRACE
-    if (p.mode == 9) { if (a[0] == 1.2345e-30f) static_cast<float *>(p.out)[0] = a[1]; return; }   // timing probe: no stores
-#endif
     if (p.mode == 0) {
         T *out = static_cast<T *>(p.out);
         const size_t plane = static_cast<size_t>(p.H) * p.W;
@@ -443,11 +430,10 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) PATDNN_STAMP(0);
     pdl_trigger();
     const int stages = p.stages;
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[8]), bar_acc = smem_u32(&bars[16]);
-    int *status = p.status;
+    const WaitCtx status{p.status, p.spin_limit ? p.spin_limit : kSpinLimit};
 
     // The ks CTAs of a cluster share one (pixel box, filter tile) and split its K loop -- the (channel block, tap)
     // iterations -- into ks ranges; then the filter tile index is fastest so that CTAs sharing a pixel box run together.
@@ -502,7 +488,6 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         }
     }
     pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
-    if (threadIdx.x == 0) PATDNN_STAMP(1);
     bool acc_ready = false;                                     // epilogue thread holding a finished K-range partial
 
     if (warp == 0) {
@@ -511,6 +496,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             for (int it = 0; it < iters; ++it) {
                 const int s = it % stages, use = it / stages;
                 if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1, status, 1)) break;
+                if (it + 1 == p.test_skip_load) continue;       // test hook: this iteration's loads never arrive
                 const int cb = (it0 + it) / p.taps, tap = (it0 + it) - cb * p.taps;
                 const int r = p.taps == 9 ? tap / 3 : 1, sx = p.taps == 9 ? tap - 3 * r : 1;
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
@@ -531,7 +517,6 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 const int s = it % stages, use = it / stages;
                 ok = mbar_wait(bar_full + 8 * s, use & 1, status, 2);
                 if (!ok) break;
-                if (it == 0) PATDNN_STAMP(2);
                 tc_fence_after();
                 const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
                 const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + A_BYTES);
@@ -553,12 +538,10 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 umma_commit(bar_empty + 8 * s);                 // frees the stage once these MMAs have read it
             }
             if (ok) umma_commit(bar_acc);
-            PATDNN_STAMP(3);
         }
     } else {
         // epilogue warps: warp w owns TMEM lanes 32*(w%4) .. +31; lane = output pixel m of the box
         if (mbar_wait(bar_acc, 0, status, 3)) {
-            if (threadIdx.x == 64) PATDNN_STAMP(4);
             tc_fence_after();
             if (ks == 1) {
 #pragma unroll 1
@@ -594,7 +577,6 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         __syncwarp();                                           // lane 0 of the two role warps rejoins its warp: the
                                                                 // cluster barriers below are warp-aligned instructions
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (threadIdx.x == 64) PATDNN_STAMP(7);
         if (acc_ready) {
 #pragma unroll 1
             for (int c0 = col_lo; c0 < col_hi; c0 += 32) {
@@ -620,9 +602,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 }
             }
         }
-        if (threadIdx.x == 64) PATDNN_STAMP(8);
         asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (threadIdx.x == 64) PATDNN_STAMP(9);
         if (warp >= 2) {
             const float4 *R4 = reinterpret_cast<const float4 *>(smem);
             const int cbeg = rank * cols;
@@ -640,12 +620,9 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 emit_chunk<8, T>(p, a, s_bias + cbeg + c0, f0 + cbeg + c0, n, y, x, pix_ok);
             }
         }
-        if (threadIdx.x == 64) PATDNN_STAMP(5);
     }
-    if (ks == 1 && threadIdx.x == 64) PATDNN_STAMP(5);
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) PATDNN_STAMP(6);
     if (warp == 2) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
@@ -690,13 +667,12 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     unsigned char *smem_b = smem + NA * a_stage;
     const uint32_t bar_fa = smem_u32(&bars[0]), bar_ea = smem_u32(&bars[8]), bar_fb = smem_u32(&bars[16]),
                    bar_eb = smem_u32(&bars[24]), bar_af = smem_u32(&bars[32]), bar_ae = smem_u32(&bars[34]);
-    int *status = p.status;
+    const WaitCtx status{p.status, p.spin_limit ? p.spin_limit : kSpinLimit};
     const int row_bytes = p.TW * 128;
     const int n_tiles = p.tile_limit > 0 ? p.tile_limit : p.n_ftiles * p.tiles_x * p.tiles_y * p.tiles_n;
     const int KB = p.KB;
     const int nshift = p.taps == 9 ? 3 : 1;                     // 3 horizontal shifts x 3 vertical taps, or one gathered tap
 
-    if (threadIdx.x == 0) PATDNN_STAMP(0);
     pdl_trigger();
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
@@ -723,7 +699,6 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         n = t; x0 = tix * p.TW; y0 = tiy * (MT * p.TH);
     };
     pdl_wait();                                                 // set-up done; from here on the previous kernel's data is read
-    if (threadIdx.x == 0) PATDNN_STAMP(1);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -766,22 +741,20 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
             int ia = 0, ib = 0, j = 0;
             bool ok = true;
-            [[maybe_unused]] long long w_fa = 0, w_fb = 0, w_ae = 0;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
                 const int buf = j & 1, ub2 = j >> 1;
-                if (ub2 > 0 && !PATDNN_TIMED(w_ae, mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2))) { ok = false; break; }
+                if (ub2 > 0 && !mbar_wait(bar_ae + 8 * buf, (ub2 - 1) & 1, status, 2)) { ok = false; break; }
                 tc_fence_after();
                 bool first = true;
                 for (int cb = 0; cb < KB && ok; ++cb) {
                     for (int sx = 0; sx < nshift && ok; ++sx) {
                         const int sa = ia % NA, ua = ia / NA;
-                        ok = PATDNN_TIMED(w_fa, mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2));
+                        ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
                         if (!ok) break;
-                        if (ia == 0) PATDNN_STAMP(2);
                         const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
                         for (int r = 0; r < nshift && ok; ++r) {
                             const int sb = ib % NB, ub = ib / NB;
-                            ok = PATDNN_TIMED(w_fb, mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2));
+                            ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
                             if (!ok) break;
                             tc_fence_after();
                             const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
@@ -817,8 +790,6 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 }
                 if (ok) umma_commit(bar_af + 8 * buf);
             }
-            PATDNN_STAMP(3);
-            PATDNN_PUT(13, w_fa); PATDNN_PUT(14, w_fb); PATDNN_PUT(15, w_ae);
         }
     } else if (GATHER && warp >= kHaloThreads / 32) {
         // gather warps: the input patch of a tile (all channels, one-pixel border, zeros outside the image) is staged
@@ -863,7 +834,6 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             if (more) fetch(t + gridDim.x);                      // loads in flight while the rows are built
             const int sa = ia % NA, ua = ia / NA;
             if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 4)) break;
-            if (g == 0 && ia == 1) PATDNN_STAMP(11);
             unsigned char *abase = smem + static_cast<size_t>(sa) * a_stage;
             for (int row = g; row < MT * kTileM; row += kGatherThreads) {
                 const int ty = row / p.TW, tx = row - ty * p.TW;
@@ -900,10 +870,8 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy writes -> visible to the MMA
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_fa + 8 * sa) : "memory");
-            if (g == 0 && ia == 1) PATDNN_STAMP(12);
             if (more) stash(patch0 + ((ia + 1) & 1) * pstride);
             asm volatile("bar.sync 2, %0;" ::"n"(kGatherThreads) : "memory");   // next patch complete, this one free
-            if (g == 0 && ia == 0) PATDNN_STAMP(9);
         }
     } else {
         // eight epilogue warps: warp w reads TMEM lanes 32*(w%4).. and one half of the filter columns
@@ -922,7 +890,6 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             asm volatile("bar.sync 1, 256;" ::: "memory");     // the eight epilogue warps only
             if (!mbar_wait(bar_af + 8 * buf, (j >> 1) & 1, status, 3)) break;
             tc_fence_after();
-            if (threadIdx.x == 64 && j == 0) PATDNN_STAMP(4);
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 const int y = y0 + mt * p.TH + ty, x = x0 + txx;
@@ -947,12 +914,10 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_ae + 8 * buf) : "memory");
-            if (threadIdx.x == 64 && j == 0) PATDNN_STAMP(5);
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) PATDNN_STAMP(6);
     if (warp == 2) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
@@ -1039,7 +1004,7 @@ conv_umma_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                    bar_eb = smem_u32(&bars[24]), bar_af = smem_u32(&bars[32]), bar_ae = smem_u32(&bars[34]);
     // the same barriers seen from the cluster: the leader's full/acc-empty barriers, each CTA's empty/acc-full barriers
     const uint32_t L_fa = map_to_cta(bar_fa, 0), L_fb = map_to_cta(bar_fb, 0), L_ae = map_to_cta(bar_ae, 0);
-    int *status = p.status;
+    const WaitCtx status{p.status, p.spin_limit ? p.spin_limit : kSpinLimit};
     const int row_bytes = p.TW * 128;
     const int pix_tiles = p.tiles_x * p.tiles_y * p.tiles_n;
     const int pair_tiles = (pix_tiles + 1) / 2;
@@ -1288,6 +1253,40 @@ cudaError_t route(const DensePlan &pl, const DenseParams &p, int dtype, cudaStre
     return cudaErrorInvalidConfiguration;
 }
 
+// CTAs of the one-tile-per-CTA kernel that are resident at the same time when launched as clusters of `ks`
+// (cudaOccupancyMaxActiveClusters; cached; the figures measured on B200 serve where the query is unavailable).
+template <int BN, int TERMS, typename T>
+int query_cluster_capacity(int ks, int smem) {
+    auto kern = conv_umma_kernel<BN, TERMS, T>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) != cudaSuccess) { cudaGetLastError(); return 0; }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ks) * 64); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ks; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n * ks;
+}
+
+int cluster_capacity(int bn, int dtype, int ks, int smem) {
+    static int cache[4][2][4] = {};                                // [BN 32..256][dtype][ks 1, 2, 4, 8], current device of first use
+    const int bi = bn == 256 ? 3 : (bn == 128 ? 2 : (bn == 64 ? 1 : 0)), ki = ks == 8 ? 3 : (ks == 4 ? 2 : (ks == 2 ? 1 : 0));
+    const int di = dtype == PATDNN_F16 ? 1 : 0;
+    if (ks <= 1) return sm_count();
+    if (cache[bi][di][ki] == 0) {
+        int n = 0;
+#define PATDNN_CAP(b)                                                                                              \
+    if (bn == b) n = di ? query_cluster_capacity<b, 1, __half>(ks, smem) : query_cluster_capacity<b, 3, float>(ks, smem);
+        PATDNN_CAP(256) PATDNN_CAP(128) PATDNN_CAP(64) PATDNN_CAP(32)
+#undef PATDNN_CAP
+        if (n <= 0) n = ks == 2 ? 148 : (ks == 4 ? 132 : 120);
+        cache[bi][di][ki] = n;
+    }
+    return cache[bi][di][ki];
+}
+
 }  // namespace
 
 bool dense_supported(int F, int C, int N, int H, int W) {
@@ -1303,8 +1302,8 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
     pl.Cp = pl.im2col ? kKBlock : (C + kKBlock - 1) / kKBlock * kKBlock;
     pl.KB = pl.Cp / kKBlock;
     pl.BN = F > 128 ? 256 : (F > 64 ? 128 : (F > 32 ? 64 : 32));
-    if (const char *bv = std::getenv("PATDNN_BN")) {             // tuning override
-        const int want = atoi(bv);
+    {
+        const int want = debug_option("bn", 0);                   // tuning override
         if (want == 32 || want == 64 || want == 128 || want == 256) pl.BN = std::min(pl.BN, want);
     }
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
@@ -1329,37 +1328,39 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
     const int ptiles = pl.tiles_x * pl.tiles_y * pl.tiles_n;
     const int total_iters = pl.taps * pl.KB;
     // a 2-way split of a 128-wide tile exchanges a quarter of what a 4-way split of a 256-wide tile does (measured faster)
-    const bool keep_bn = std::getenv("PATDNN_BN_KEEP") != nullptr;   // tuning override: no narrowing
-    while (!keep_bn && pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 < 100) pl.BN /= 2;
-    while (!keep_bn && pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 8 < 60) pl.BN /= 2;   // 8-way split still too few CTAs
+    const bool keep_bn = debug_option("bn_keep", 0) != 0;        // tuning override: no narrowing
+    const int n_sm0 = sm_count();
+    while (!keep_bn && pl.BN > 128 && ptiles * ((F + pl.BN - 1) / pl.BN) * 2 * 37 < n_sm0 * 25) pl.BN /= 2;
+    while (!keep_bn && pl.BN > 64 && ptiles * ((F + pl.BN - 1) / pl.BN) * 8 * 37 < n_sm0 * 15) pl.BN /= 2;   // 8-way split still too few CTAs
     if (force_bn) pl.BN = force_bn;
     pl.poolable = (pool_tiles && best > 0) ? 1 : 0;
     pl.Fp = (F + pl.BN - 1) / pl.BN * pl.BN;
     pl.n_ftiles = pl.Fp / pl.BN;
     const int base_grid = ptiles * pl.n_ftiles;
+    const int stage = pl.S * (kTileM * 128 + pl.BN * 128);
+    pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
+    pl.smem_bytes = pl.stages * stage + 1024;
+    const int n_sm = sm_count();
     int ks = 1;
-    // one wave only: with ~200 KB of shared memory per CTA, 148 CTAs fit as clusters of 2, 132 as clusters of 4, 120 as
-    // clusters of 8 (occupancy query); a second wave costs more than the shorter loop saves
-    if (base_grid < 100)
-        while (ks < 8 && base_grid * ks * 2 <= (ks * 2 == 2 ? 148 : (ks * 2 == 4 ? 132 : 120)) && ks * 2 <= total_iters &&
+    // one wave only: a second wave costs more than the shorter loop saves.  How many CTAs of this kernel are resident
+    // at once as clusters of 2, 4 or 8 comes from the occupancy query (B200, ~200 KB of shared memory per CTA: 148 / 132 / 120)
+    if (base_grid * 37 < n_sm * 25)                            // fewer CTAs than about two thirds of the SMs
+        while (ks < 8 && base_grid * ks * 2 <= cluster_capacity(pl.BN, dtype, ks * 2, pl.smem_bytes) && ks * 2 <= total_iters &&
                pl.BN / (ks * 2) >= 8)
             ks *= 2;
-    if (const char *ov = std::getenv("PATDNN_KSPLIT")) {
-        const int want = atoi(ov);
+    {
+        const int want = debug_option("ksplit", 0);
         if ((want == 1 || want == 2 || want == 4 || want == 8) && want <= total_iters && pl.BN / want >= 8) ks = want;
     }
     pl.ksplit = ks;
     pl.iters_per_split = (total_iters + ks - 1) / ks;
     pl.box_bytes = pl.TW * pl.TH * pl.TN * 128;
-    const int stage = pl.S * (kTileM * 128 + pl.BN * 128);
-    pl.stages = std::max(2, std::min(8, (220 * 1024) / stage));
-    pl.smem_bytes = pl.stages * stage + 1024;
     pl.grid = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles * pl.ksplit;
 
     // Large grids: the halo-sharing kernel (three boxes per channel block instead of nine) if a TW x TH = 128 box
     // with TW a multiple of 8 wastes no more pixels than the free-form box does.
-    const char *hv = std::getenv("PATDNN_HALO");
-    if (pl.ksplit == 1 && pl.BN >= 64 && !(hv && hv[0] == '0')) {
+    const bool halo_ok = debug_option("halo", 1) != 0;
+    if (pl.ksplit == 1 && pl.BN >= 64 && halo_ok) {
         const double util_now = static_cast<double>(N) * H * W / (static_cast<double>(ptiles) * kTileM);
         int btw = 0; double butil = 0;
         for (int tw : {32, 16, 8, 64, 128}) {                      // ties: 32-wide boxes first (128-byte store rows, 1.5x halo)
@@ -1379,10 +1380,10 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             if (mt == 2) {
                 // a double tile costs ~1/0.65 single tiles (measured); with few rounds the finer granularity can win
                 const long long t1 = static_cast<long long>((W + btw - 1) / btw) * ((H + th - 1) / th) * N * pl.n_ftiles;
-                const long long r1 = (t1 + 147) / 148, r2 = (t1 / 2 + 147) / 148;
+                const long long r1 = (t1 + n_sm - 1) / n_sm, r2 = (t1 / 2 + n_sm - 1) / n_sm;
                 if (0.65 * static_cast<double>(r1) < static_cast<double>(r2)) mt = 1;
             }
-            if (const char *mv = std::getenv("PATDNN_MT")) mt = (atoi(mv) == 2 && pl.BN == 64) ? 2 : 1;
+            if (const int mv = debug_option("mt", 0)) mt = (mv == 2 && pl.BN == 64) ? 2 : 1;
             const int hr = pl.im2col ? 0 : 2;
             const int a_stage = pl.S * (mt * th + hr) * btw * 128;
             const int b_stage = pl.S * pl.BN * 128;
@@ -1401,16 +1402,15 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
                 pl.na = na; pl.stages = nb;
                 pl.smem_bytes = na * a_stage + nb * b_stage + patch + 1024;
                 pl.n_tiles = pl.tiles_x * pl.tiles_y * pl.tiles_n * pl.n_ftiles;
-                pl.grid = std::min(pl.n_tiles, 148);             // persistent CTAs, one per SM
+                pl.grid = std::min(pl.n_tiles, n_sm);            // persistent CTAs, one per SM
             }
         }
     }
     // 256-filter tiles with enough pixel tiles: CTA pairs (cta_group::2), each CTA loading half of every weight tile.
-    // Half-size weight stages also let the 28-pixel-wide halo boxes fit.  Opt-in (PATDNN_PAIR=1): correct, but measured
+    // Half-size weight stages also let the 28-pixel-wide halo boxes fit.  Opt-in (PATDNN_DEBUG=pair=1): correct, but measured
     // 8-12 % slower than the single-CTA kernels on the 56x56 and 28x28 layers at batch 32 -- those are not bound by the
     // weight traffic this halves.
-    const char *pv = std::getenv("PATDNN_PAIR");
-    if (pl.BN == 256 && pl.ksplit == 1 && !pl.im2col && !pool_tiles && pv && pv[0] == '1' && !(hv && hv[0] == '0')) {
+    if (pl.BN == 256 && pl.ksplit == 1 && !pl.im2col && !pool_tiles && debug_option("pair", 0) == 1 && halo_ok) {
         const double util_free = static_cast<double>(N) * H * W / (static_cast<double>(ptiles) * kTileM);
         int btw = 0; double butil = 0;
         for (int tw : {32, 16, 8}) {
@@ -1425,7 +1425,7 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             const int tx = (W + btw - 1) / btw, ty = (H + th - 1) / th;
             const int pix_tiles = tx * ty * N;
             const int n_pairs = ((pix_tiles + 1) / 2) * pl.n_ftiles;
-            if (n_pairs >= 74) {
+            if (n_pairs >= n_sm / 2) {
                 const int a_stage = pl.S * (th + 2) * btw * 128, b_stage = pl.S * 128 * 128;
                 int na = 2, nb = 2;
                 const int budget = 218 * 1024;
@@ -1437,30 +1437,29 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
                 pl.na = na; pl.stages = nb;
                 pl.smem_bytes = na * a_stage + nb * b_stage + 1024;
                 pl.n_tiles = n_pairs;                            // pair tiles
-                pl.grid = 2 * std::min(n_pairs, 74);
+                pl.grid = 2 * std::min(n_pairs, n_sm / 2);
                 pl.tail_tiles = 0;
                 return;
             }
         }
     }
-    // Round quantisation: T equal tiles on 148 SMs take ceil(T/148) rounds.  When the last round is nearly empty its
+    // Round quantisation: T equal tiles on n_sm SMs take ceil(T/n_sm) rounds.  When the last round is nearly empty its
     // tiles go to a second launch whose K loop is split over clusters (largest split that still fits one wave).
-    const char *tv = std::getenv("PATDNN_TAIL");
     const int T = pl.halo ? pl.n_tiles : pl.grid;
-    if (!(tv && tv[0] == '0') && pl.ksplit == 1 && pl.MT == 1 && !pl.gather && T > 148 && T % 148 != 0) {
-        const int tail = T % 148;
+    if (debug_option("tail", 1) != 0 && pl.ksplit == 1 && pl.MT == 1 && !pl.gather && T > n_sm && T % n_sm != 0) {
+        const int tail = T % n_sm;
+        const int tstage = pl.S * (kTileM * 128 + pl.BN * 128);
+        const int tstages = std::max(2, std::min(8, (220 * 1024) / tstage));
+        const int tsmem = tstages * tstage + 1024;
         int tks = 0;
-        for (int cand : {8, 4, 2}) {
-            const int cap = cand == 8 ? 120 : (cand == 4 ? 132 : 148);
-            if (tail * cand <= cap && total_iters / cand >= 2 && pl.BN / cand >= 8) { tks = cand; break; }
-        }
+        for (int cand : {8, 4, 2})
+            if (tail * cand <= cluster_capacity(pl.BN, dtype, cand, tsmem) && total_iters / cand >= 2 && pl.BN / cand >= 8) { tks = cand; break; }
         if (tks) {
             pl.tail_tiles = tail; pl.tail_ks = tks;
-            const int tstage = pl.S * (kTileM * 128 + pl.BN * 128);
-            pl.tail_stages = std::max(2, std::min(8, (220 * 1024) / tstage));
-            pl.tail_smem = pl.tail_stages * tstage + 1024;
+            pl.tail_stages = tstages;
+            pl.tail_smem = tsmem;
             pl.tail_box_bytes = pl.TW * pl.TH * pl.TN * 128;
-            if (pl.halo) pl.grid = std::min(T - tail, 148);
+            if (pl.halo) pl.grid = std::min(T - tail, n_sm);
             else pl.grid = T - tail;
         }
     }
@@ -1548,27 +1547,23 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // Device address of g_static_scratch for the current device.  In host code the symbol is only a handle, not an
-// address a kernel can use: the address comes from cudaGetSymbolAddress, once per device.
-int static_scratch_address(void **ptr) {
+// address a kernel can use: the address comes from cudaGetSymbolAddress, once per device (the caller serialises).
+cudaError_t static_scratch_address(void **ptr) {
     static void *addr[64] = {};
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess || dev < 0 || dev >= 64) return PATDNN_E_CUDA;
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!addr[dev]) {
         void *p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (e != cudaSuccess || !p) return PATDNN_E_CUDA;
+        if (e != cudaSuccess) return e;
+        if (!p) return cudaErrorInvalidSymbol;
         addr[dev] = p;
     }
     *ptr = addr[dev];
-    return PATDNN_OK;
+    return cudaSuccess;
 }
-
-#ifdef PATDNN_TRACE
-extern "C" __attribute__((visibility("default"))) int patdnn_trace_read(unsigned long long *host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(unsigned long long) * n);
-}
-#endif
 
 cudaError_t prepare_dense(const DensePlan &pl, int dtype) {
     DenseParams dummy{};

@@ -144,3 +144,28 @@ def test_index_structure_is_far_smaller_than_csr():
     assert 1 - b["fkw_index"] / b["csr_index"] > 0.70
     b16 = fkw_ref.storage_bytes(F, C, K, 8, index_bytes=2)
     assert b16["fkw_index"] * 2 == b["fkw_index"]
+
+
+def test_storage_saving_with_the_widths_that_fit_section_6_4():
+    """Section 6.4 prints 93.4 % (index) and 46.7 % (total) saved at 18x.  One byte of index per kept kernel against
+    four bytes per weight in CSR gives 1 - 1/16 and 1 - 17/32 when the per-filter arrays are negligible; the
+    function must reach those closed forms from below as filters get longer, and the 18x layer must sit near them."""
+    P = 8
+    last = 0.0
+    for per_filter in (16, 64, 256, 4096, 1 << 16):
+        F = 8
+        b = fkw_ref.storage_bytes(F, per_filter * 4, F * per_filter, P, index_bytes=1, filter_bytes=2, csr_index_bytes=4)
+        idx = 1 - b["fkw_index"] / b["csr_index"]
+        tot = 1 - (b["fkw_index"] + b["weights"]) / (b["csr_index"] + b["weights"])
+        assert last < idx < 15 / 16 and tot < 15 / 32
+        last = idx
+    assert abs(idx - 15 / 16) < 1e-3 and abs(tot - 15 / 32) < 1e-3
+    # by hand for a tiny case: F = 2 filters, K = 3 kernels, P = 2 patterns
+    b = fkw_ref.storage_bytes(2, 4, 3, 2, index_bytes=1, filter_bytes=2, csr_index_bytes=4)
+    assert b["fkw_index"] == 3 * 2 + 2 * 2 + 3 * 1 + 2 * 3 * 2          # offset[3], reorder[2], index[3], stride[2][3]
+    assert b["csr_index"] == 3 * 4 + 12 * 4 and b["weights"] == 48
+    # 512 x 512 layer at an overall rate of 18x: 64 kernels per filter
+    b = fkw_ref.storage_bytes(512, 512, 512 * 64, P, index_bytes=1, filter_bytes=2, csr_index_bytes=4)
+    idx = 1 - b["fkw_index"] / b["csr_index"]
+    assert 0.90 < idx < 0.9375                                            # the paper prints 93.4 %
+

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from paper_2001_00138_b200 import build, synth
-from util import TOL_F16, TOL_F32, assert_close, gpu_layer, oracle_layer
+from util import TOL_F16, TOL_F32, assert_close, chain_tol, gpu_layer, oracle_layer
 
 pytestmark = pytest.mark.gpu
 
@@ -100,11 +100,14 @@ def test_config2_full_size():
 
 
 @pytest.mark.parametrize("i", range(4))
-@pytest.mark.parametrize("N", [1, 3])
+@pytest.mark.parametrize("N", [1, 3, 32])
 def test_resnet_shapes_fp16(i, N):
+    """The four ResNet-50-shaped fp16 layers at batch 1, a ragged batch and the full batch of 32, whole output."""
     L = synth.resnet50_layer(i, N=N)
     ref = oracle_layer(L)
     for variant in ("auto", "tiled", "dense", "reorder"):
+        if N == 32 and variant == "reorder":
+            continue                      # the generic kernel adds nothing at full batch
         if variant == "tiled" and L.W % 2:
             continue                      # odd-width fp16 rows are not 4-byte aligned: no tiled kernel for them
         got, _ = gpu_layer(L, variant=VARIANTS[variant])
@@ -140,7 +143,7 @@ def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype, g
     from paper_2001_00138_b200 import binding as B
     N, C, F, H, W = shape
     if not generated:
-        monkeypatch.setenv("PATDNN_NO_JIT", "1")
+        monkeypatch.setenv("PATDNN_DEBUG", "jit=0")
     dt = B.F16 if dtype == "f16" else B.F32
     tdt = torch.float16 if dtype == "f16" else torch.float32
     L0 = synth.make_layer("f0", F=F, C=C, N=N, H=H, W=W, seed=77 + C, prune=0.0, bias_std=0.3, x_dist="normal", dtype=dtype)
@@ -158,7 +161,8 @@ def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype, g
     stack.run(torch.from_numpy(L0.x).to("cuda", dtype=tdt), out, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert B.launch_count() == 2
-    assert_close(out.float().cpu().numpy(), ref, 3 * (TOL_F16 if dtype == "f16" else TOL_F32), f"fused first layer {shape} {dtype}")
+    assert_close(out.float().cpu().numpy(), ref, chain_tol(2, TOL_F16 if dtype == "f16" else TOL_F32),
+                 f"fused first layer {shape} {dtype}")
     stack.free()
     h0.free()
     h1.free()
@@ -173,6 +177,19 @@ def test_sweep_points_reduced_batch(npat, prune):
         assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune} {variant}")
     got, _ = gpu_layer(L, order=synth.random_filter_order(512, 1))
     assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune} random filter order")
+
+
+@pytest.mark.parametrize("npat,prune", [(4, 0.9), (6, 0.75), (8, 0.0), (12, 0.5), (8, 0.9)])
+def test_sweep_points_full_batch(npat, prune):
+    """Sweep points at the full batch of 64 (the launch configuration the sweep is timed in), whole output, with the
+    filter reorder and with a seeded random filter order."""
+    L = synth.sweep_layer(npat, prune, N=64)
+    ref = oracle_layer(L)
+    for variant in ("auto", "tiled"):
+        got, _ = gpu_layer(L, variant=VARIANTS[variant])
+        assert_close(got, ref, TOL_F32, f"sweep N=64 p{npat} prune{prune} {variant}")
+    got, _ = gpu_layer(L, order=synth.random_filter_order(512, 7))
+    assert_close(got, ref, TOL_F32, f"sweep N=64 p{npat} prune{prune} random filter order")
 
 
 @pytest.mark.parametrize("scale,N", [(4, 2), (7, 5)])
@@ -201,10 +218,11 @@ def test_vgg_stack_reduced_spatial_per_layer_and_chained(scale, N):
     out = torch.empty(cur.shape, device="cuda")
     stack.run(xt, out, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
-    assert_close(out.cpu().numpy(), cur, 10 * TOL_F32, "vgg chained")      # 13 layers of rounding compound
+    assert_close(out.cpu().numpy(), cur, chain_tol(13, TOL_F32), "vgg chained")
     out_h = np.empty(cur.shape, dtype=np.float32)
     stack.run_host(x, out_h)
-    assert_close(out_h, cur, 10 * TOL_F32, "vgg chained through host buffers")   # K-split sums are order-free
+    # same kernels, and the cluster reduction of K-split partial tiles adds in rank order: the same bits
+    assert np.array_equal(out_h, out.cpu().numpy()), "vgg chained through host buffers"
     stack.free()
     for h in handles:
         h.free()
@@ -212,7 +230,7 @@ def test_vgg_stack_reduced_spatial_per_layer_and_chained(scale, N):
 
 @pytest.mark.parametrize("variants", [("dense", "dense", "dense"), ("tiled", "dense", "tiled"), ("dense", "tiled", "dense"),
                                       ("reorder", "dense", "dense")])
-@pytest.mark.parametrize("hw", [(7, 7), (13, 9), (6, 10), (5, 3)])
+@pytest.mark.parametrize("hw", [(7, 7), (13, 9), (6, 10), (5, 7)])
 def test_small_stack_with_odd_sizes_and_pools(variants, hw):
     """Three chained layers with a pool after the first two, on extents that are odd before and after pooling, with
     every hand-over between the kernel families (NCHW <-> channels-innermost split operands, pooled or not)."""
@@ -233,8 +251,7 @@ def test_small_stack_with_odd_sizes_and_pools(variants, hw):
             cur = oracle.maxpool2x2(cur)
             h, w = h // 2, w // 2
     pools = [1 if (i < 2) else 0 for i in range(3)]
-    if cur.shape[2:] != (h, w) or H // 2 // 2 < 1 or W // 2 // 2 < 1:
-        pytest.skip("extent too small for two pools")
+    assert cur.shape[2:] == (h, w) and h >= 1 and w >= 1
     stack = B.Stack(handles, pools)
     assert stack.out_shape() == cur.shape
     out = torch.empty(cur.shape, device="cuda")
@@ -245,16 +262,16 @@ def test_small_stack_with_odd_sizes_and_pools(variants, hw):
         # three GEMMs, both pools taken in their epilogues; the first layer (9*C <= 64) either gathers its operand rows
         # from the caller's NCHW input itself or has one layout kernel in front
         assert B.launch_count() in (3, 4)
-    assert_close(out.cpu().numpy(), cur, 4 * TOL_F32, f"stack {variants} {hw}")
+    assert_close(out.cpu().numpy(), cur, chain_tol(3, TOL_F32), f"stack {variants} {hw}")
     stack.free()
     for hd in handles:
         hd.free()
 
 
-@pytest.mark.parametrize("i,N", [(0, 32), (1, 32), (5, 32), (8, 32), (12, 32), (3, 1), (8, 1), (11, 1)])
-def test_vgg_full_size_sampled(i, N):
-    """Full-size layers in the benchmark's launch configuration; outputs sampled and checked one by one."""
-    import oracle
+@pytest.mark.parametrize("i,N", [(0, 32), (1, 32), (2, 32), (5, 32), (8, 32), (12, 32), (3, 1), (8, 1), (11, 1)])
+def test_vgg_full_size_standalone(i, N):
+    """Full-size layers called alone (NCHW in, NCHW out) in the benchmark's launch configuration; the whole output is
+    compared with the oracle."""
     import torch
     from paper_2001_00138_b200 import binding as B
     L = synth.vgg16_layer(i, N=N)
@@ -264,30 +281,21 @@ def test_vgg_full_size_sampled(i, N):
     xt = torch.from_numpy(x).cuda()
     out = torch.full((N, L.F, L.H, L.W), float("nan"), device="cuda")
     layer.conv(xt, out, torch.cuda.current_stream().cuda_stream)
-    torch.cuda.synchronize()
-    assert bool(torch.isfinite(out).all())
+    layer.check()
     got = out.cpu().numpy()
-    pts = [(0, 0, 0, 0), (N - 1, L.F - 1, L.H - 1, L.W - 1), (N - 1, 0, 0, L.W - 1), (0, L.F - 1, L.H - 1, 0)]
-    for _ in range(300):
-        pts.append((int(rng.integers(N)), int(rng.integers(L.F)), int(rng.integers(L.H)), int(rng.integers(L.W))))
-    for _ in range(60):     # the last image holds the tiles of a K-split tail launch, where the plan has one
-        pts.append((N - 1, int(rng.integers(L.F)), int(rng.integers(L.H)), int(rng.integers(L.W))))
     if i == 0:
         assert layer.plan()["generated"] == 1, "the RGB layer under AUTO runs code generated for it"
     if (i, N) in ((5, 32), (8, 32)):
-        assert layer.plan()["grid_z"] > 1, "these tile counts are not whole rounds of 148 CTAs: a tail launch is planned"
-    ref = np.asarray([oracle.conv3x3_point(x, L.weights, L.mask, L.bias, True, *p) for p in pts])
-    vals = np.asarray([got[p] for p in pts])
-    rms = float(np.sqrt(np.mean(got.astype(np.float64) ** 2)))
-    assert np.all(np.abs(vals - ref) <= TOL_F32 * np.maximum(np.abs(ref), rms)), f"vgg L{i + 1} N={N}"
+        assert layer.plan()["grid_z"] > 1, "these tile counts are not whole rounds of CTAs: a tail launch is planned"
     layer.free()
+    assert_close(got, oracle_layer(L, x=x), TOL_F32, f"vgg L{i + 1} N={N}")
 
 
 @pytest.mark.parametrize("ks", [1, 2, 4, 8])
 def test_tensor_core_path_with_cluster_split_of_the_channel_loop(ks, monkeypatch):
     """Small batches split the (channel block, tap) loop over the CTAs of a cluster and sum through distributed shared
     memory; every split factor must give the same layer."""
-    monkeypatch.setenv("PATDNN_KSPLIT", str(ks))
+    monkeypatch.setenv("PATDNN_DEBUG", f"ksplit={ks}")
     L = synth.make_layer("ks", F=192, C=160, N=1, H=20, W=24, seed=900 + ks, prune=0.6, bias_std=0.1, x_dist="normal")
     got, plan = gpu_layer(L, variant=VARIANTS["dense"])
     assert plan["variant"] == 4
@@ -377,7 +385,7 @@ def test_fp16_stack_with_pools(hw):
     torch.cuda.synchronize()
     for hd in handles:
         hd.check()
-    assert_close(out.float().cpu().numpy(), cur, 4 * TOL_F16, f"fp16 stack {hw}")
+    assert_close(out.float().cpu().numpy(), cur, chain_tol(4, TOL_F16), f"fp16 stack {hw}")
     stack.free()
     for hd in handles:
         hd.free()
@@ -402,7 +410,7 @@ def test_cta_pair_kernel(shape, monkeypatch):
     layer as the default kernels, odd pixel-tile counts and padded filter tiles included."""
     import torch
     from paper_2001_00138_b200 import binding as B
-    monkeypatch.setenv("PATDNN_PAIR", "1")
+    monkeypatch.setenv("PATDNN_DEBUG", "pair=1")
     N, C, F, H, W = shape
     L = synth.make_layer("pair", F=F, C=C, N=N, H=H, W=W, seed=N + F, prune=0.6, bias_std=0.2, draw_input=False,
                          w_std=float(np.sqrt(2.0 / (4 * C * 0.4))))
@@ -415,15 +423,8 @@ def test_cta_pair_kernel(shape, monkeypatch):
     layer.conv(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
     layer.check()
     got = out.cpu().numpy()
-    assert np.all(np.isfinite(got))
     import oracle
-    pts = [(0, 0, 0, 0), (N - 1, F - 1, H - 1, W - 1), (N - 1, 0, H - 1, 0), (0, F - 1, 0, W - 1)]
-    for _ in range(250):
-        pts.append((int(rng.integers(N)), int(rng.integers(F)), int(rng.integers(H)), int(rng.integers(W))))
-    ref = np.asarray([oracle.conv3x3_point(x, L.weights, L.mask, L.bias, True, *pt) for pt in pts])
-    vals = np.asarray([got[pt] for pt in pts])
-    rms = float(np.sqrt(np.mean(got.astype(np.float64) ** 2)))
-    assert np.all(np.abs(vals - ref) <= TOL_F32 * np.maximum(np.abs(ref), rms))
+    assert_close(got, oracle.conv3x3(x, L.weights, L.mask, L.bias, True), TOL_F32, f"CTA-pair kernel {shape}")
     layer.free()
 
 
@@ -491,7 +492,7 @@ def test_random_stacks(seed):
     torch.cuda.synchronize()
     for hd in handles:
         hd.check()
-    assert_close(out.cpu().numpy(), cur, 5 * TOL_F32, f"random stack {seed}: {chans} pools {pools} {H}x{W} N={N}")
+    assert_close(out.cpu().numpy(), cur, chain_tol(nl, TOL_F32), f"random stack {seed}: {chans} pools {pools} {H}x{W} N={N}")
     stack.free()
     for hd in handles:
         hd.free()

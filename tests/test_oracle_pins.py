@@ -144,10 +144,24 @@ def test_point_function_agrees_with_full_tensor():
         assert np.float32(oracle.conv3x3_point(x, w, mask, bias, True, n, f, y, xx)) == full[n, f, y, xx]
 
 
-def test_maxpool_matches_library():
-    x = np.random.Generator(np.random.PCG64(6)).standard_normal((2, 3, 6, 8)).astype(np.float32)
+@pytest.mark.parametrize("hw", [(6, 8), (7, 9), (5, 3), (13, 9), (2, 2), (3, 2), (14, 15)])
+def test_maxpool_matches_library(hw):
+    """2x2 / stride-2 maximum with floor extents: an odd last row or column is dropped, as the library pool does."""
+    H, W = hw
+    x = np.random.Generator(np.random.PCG64(6 + H * W)).standard_normal((2, 3, H, W)).astype(np.float32)
     ref = torch.nn.functional.max_pool2d(torch.from_numpy(x), 2).numpy()
-    assert np.array_equal(oracle.maxpool2x2(x), ref)
+    got = oracle.maxpool2x2(x)
+    assert got.shape == (2, 3, H // 2, W // 2)
+    assert np.array_equal(got, ref)
+
+
+def test_maxpool_closed_form_on_a_ramp():
+    """On a ramp that grows along rows and columns every window's maximum is its bottom-right element."""
+    H, W = 7, 5
+    x = (np.arange(H)[:, None] * 100 + np.arange(W)[None, :]).astype(np.float32).reshape(1, 1, H, W)
+    got = oracle.maxpool2x2(x)[0, 0]
+    exp = x[0, 0, 1:2 * (H // 2):2, 1:2 * (W // 2):2]
+    assert np.array_equal(got, exp)
 
 
 def test_threads_do_not_change_the_result():

@@ -50,3 +50,25 @@ def gpu_layer(L, x=None, variant=0, order=None, via_host=False):
         return out.float().cpu().numpy(), layer.plan()
     finally:
         layer.free()
+
+
+def chain_tol(n_layers: int, tol: float) -> float:
+    """Bound for a chain of n_layers compared with the chained oracle.  The chains of these tests are He-scaled (an
+    input perturbation passes a layer with rms gain of about one) and each layer's measured error is a small fraction
+    of its allowance, so the chained results are held to the single-layer tolerance as well."""
+    return tol
+
+
+def identity_layer(F: int):
+    """(weights, mask, patterns) of a C = F layer that copies its input: one kept kernel per filter, on the channel
+    of the same number, whose pattern's centre weight is 1.0 and whose other three kept weights are 0.0."""
+    from paper_2001_00138_b200 import synth
+    pats = synth.pattern_set(8)
+    taps = synth.mask_to_taps(int(pats[0]))
+    w = np.zeros((F, F, 3, 3), dtype=np.float32)
+    m = np.zeros((F, F, 3, 3), dtype=np.uint8)
+    for f in range(F):
+        for t in taps:
+            m[f, f, t // 3, t % 3] = 1
+        w[f, f, 1, 1] = 1.0
+    return w, m, pats
