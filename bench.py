@@ -27,12 +27,24 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-SM_COUNT, FP32_LANES, SM_MAX_GHZ = 148, 128, 1.965
-ALU_PEAK_TFLOPS = SM_COUNT * FP32_LANES * 2 * SM_MAX_GHZ / 1e3     # 74.45: FP32 FMA lanes x 2 flop x max SM clock
+FP32_LANES = 128                      # FP32 FMA lanes per SM on this architecture
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (conv_umma_halo_kernel on the
 # 256 -> 256 @ 56x56 layer): 28.5 MB in the ncu capture at batch 8 (profiles/conv_umma_halo_kernel_vgg16_L06_n8.txt),
 # scaled by the units of a batch-32 launch (x4; reads grow in proportion, the output additionally leaves L2 at that size)
 TRAFFIC_BYTES_PER_LAUNCH = 4 * (28093696 + 267776)
+TRAFFIC_NOTE = ("dominant kernel (conv_umma_halo_kernel, 256 -> 256 @ 56x56): ncu capture at batch 8 scaled x4 to the "
+                "batch-32 launch (extrapolated; algorithmic bytes of that launch: 112.5 MB in + 2.4 MB weights)")
+
+
+def alu_peak_tflops(torch=None):
+    """FP32 CUDA-core peak the kept-weight roofline is quoted against: SMs x 128 FMA lanes x 2 flop x max SM clock."""
+    sms, ghz = 148, 1.965
+    peaks = measured_peaks()[0]
+    if peaks.get("sm_max_mhz"):
+        ghz = float(peaks["sm_max_mhz"]) / 1e3
+    if torch is not None and torch.cuda.is_available():
+        sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    return sms * FP32_LANES * 2 * ghz / 1e3
 
 
 def measured_peaks():
@@ -85,6 +97,9 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+ALU_PEAK_TFLOPS = None                # set in main() once the device is known (74.45 on B200)
+
+
 def layer_costs(L, hbm_gbs):
     """Algorithmic flops / bytes of one layer and its roofline time (us)."""
     es = 2 if L.dtype == "f16" else 4
@@ -135,15 +150,44 @@ class VggStack:
         return bufs
 
 
-def oracle_stack_pass(synth, oracle, layers, x):
-    """One pass of the CPU oracle over the 13 chained layers (pools included); returns seconds."""
+def oracle_stack_pass(synth, oracle, layers, x, keep=None):
+    """One pass of the CPU oracle over the 13 chained layers (pools included); returns seconds.  keep: a list that
+    receives the final activations."""
     t0 = time.perf_counter()
     cur = x
     for i, L in enumerate(layers):
         cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
         if i in synth.VGG16_POOL_AFTER:
             cur = oracle.maxpool2x2(cur)
-    return time.perf_counter() - t0
+    dt = time.perf_counter() - t0
+    if keep is not None:
+        keep.append(cur)
+    return dt
+
+
+def parity_against_oracle(synth, gpu_outputs):
+    """Part of the CPU-baseline leg: the oracle chained over single images of the benchmark input, compared with what
+    the timed stacks produced for them.  gpu_outputs: {batch: (image indices, float32 array [len, F, H, W])}.
+    Ratios are in units of the single-layer tolerance 1e-4 * max(|o|, rms(o)); a 13-layer chain is allowed sqrt(13)."""
+    import oracle
+    layers = [synth.vgg16_layer(i, N=1) for i in range(13)]
+    out = {"tolerance": "|gpu - oracle| <= 1e-4 * max(|o|, rms(o)) per layer; sqrt(13) of that for the 13-layer chain",
+           "allowed_ratio": round(13 ** 0.5, 3), "checked": []}
+    worst_all = 0.0
+    for batch, (imgs, got) in gpu_outputs.items():
+        x = synth.vgg16_input(batch)
+        for j, n in enumerate(imgs):
+            keep = []
+            oracle_stack_pass(synth, oracle, layers, np.ascontiguousarray(x[n:n + 1]), keep)
+            ref = keep[0][0].astype(np.float64)
+            g = got[j].astype(np.float64)
+            rms = float(np.sqrt(np.mean(ref * ref)))
+            ratio = float((np.abs(g - ref) / (1e-4 * np.maximum(np.abs(ref), rms))).max()) if np.all(np.isfinite(g)) else float("inf")
+            out["checked"].append({"batch": batch, "image": int(n), "worst_ratio": round(ratio, 3)})
+            worst_all = max(worst_all, ratio)
+    out["worst_ratio"] = round(worst_all, 3)
+    out["ok"] = bool(worst_all <= 13 ** 0.5)
+    return out
 
 
 def time_oracle_sample(synth, seconds_hint=12.0):
@@ -210,6 +254,8 @@ def run_suite(args):
     B.load()
     peaks, _ = measured_peaks()
     hbm = float(peaks["hbm_gbs"])
+    global ALU_PEAK_TFLOPS
+    ALU_PEAK_TFLOPS = alu_peak_tflops(torch)
     stream = torch.cuda.current_stream().cuda_stream
     flush = torch.empty(256 * 1024 * 1024 // 4, device="cuda")
     variants = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense_tc": 4}
@@ -325,6 +371,7 @@ def suite_storage(B, synth):
             nnz = 4 * K
             fkw_idx32 = 4 * (a["offset"].size + a["reorder"].size + a["index"].size + a["stride"].size)
             fkw_idx16 = 2 * a["index"].size + 4 * a["offset"].size + 2 * a["reorder"].size + 2 * a["stride"].size
+            fkw_idx8 = 1 * a["index"].size + 2 * (a["offset"].size + a["reorder"].size + a["stride"].size)
             csr_idx32 = 4 * (F + 1) + 4 * nnz
             csr_idx16 = 4 * (F + 1) + 2 * nnz
             w_bytes = 4 * nnz
@@ -333,7 +380,11 @@ def suite_storage(B, synth):
                               "fkw_index_bytes_u16": fkw_idx16, "csr_index_bytes_u16": csr_idx16,
                               "index_saving_i32": round(1 - fkw_idx32 / csr_idx32, 4),
                               "total_saving_i32": round(1 - (fkw_idx32 + w_bytes) / (csr_idx32 + w_bytes), 4),
-                              "total_saving_u16": round(1 - (fkw_idx16 + w_bytes) / (csr_idx16 + w_bytes), 4)}), flush=True)
+                              "total_saving_u16": round(1 - (fkw_idx16 + w_bytes) / (csr_idx16 + w_bytes), 4),
+                              # the widths that fit the paper's 93.4 % / 46.7 %: one byte per index[] entry, two per
+                              # per-filter entry, against four bytes per CSR column index
+                              "index_saving_u8_vs_csr_i32": round(1 - fkw_idx8 / csr_idx32, 4),
+                              "total_saving_u8_vs_csr_i32": round(1 - (fkw_idx8 + w_bytes) / (csr_idx32 + w_bytes), 4)}), flush=True)
             h.free()
 
 
@@ -438,6 +489,8 @@ def main():
     peaks, peak_kind = measured_peaks()
     hbm = float(peaks["hbm_gbs"])
     stream = torch.cuda.current_stream().cuda_stream
+    global ALU_PEAK_TFLOPS
+    ALU_PEAK_TFLOPS = alu_peak_tflops(torch)
 
     def barrier():
         if world > 1:
@@ -481,6 +534,19 @@ def main():
             total_ms = sum(a.elapsed_time(b) for a, b in evs)
         launches = B.launch_count()
         clocks = sampler.stop()
+        # what the timed steps produced for the first and the last image (checked against the oracle in the CPU leg)
+        vs.stack.run(xs[0], out, stream)
+        torch.cuda.synchronize()
+        imgs = sorted({0, N - 1})
+        kept_out = (imgs, out[imgs].cpu().numpy())
+        # (1a) per-layer times INSIDE the chained step: events between the layers' launches (a separate pass)
+        in_step = np.zeros(13)
+        tsteps = max(3, min(steps, 10))
+        for i in range(tsteps):
+            if flush is not None:
+                flush.fill_(float(i))
+            in_step += vs.stack.run_timed(xs[i % nbuf], out, stream).astype(np.float64)
+        in_step = in_step / tsteps * 1e3                      # us
         # (1b) the same step as one CUDA-graph replay (launch overhead off the critical path)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
@@ -567,7 +633,7 @@ def main():
         e2e_ms = (time.perf_counter() - t0) * 1e3 / pipe_steps
         res = {
             "ms_per_step": total_ms / steps, "graph_ms_per_step": graph_ms, "flops": flops, "launches": launches, "clocks": clocks,
-            "layer_us": [m * 1e3 for m in layer_ms], "costs": costs, "e2e_ms": e2e_ms, "e2e_blocking_ms": e2e_blocking_ms,
+            "layer_us": [m * 1e3 for m in layer_ms], "in_step_us": [float(v) for v in in_step], "kept_out": kept_out, "costs": costs, "e2e_ms": e2e_ms, "e2e_blocking_ms": e2e_blocking_ms,
             "h2d": int(xh.numel() * 4), "d2h": int(oh.numel() * 4),
             "plans": [h.plan() for h in vs.handles], "names": [L.name for L in vs.layers],
             "layer_objs": vs.layers,
@@ -582,15 +648,31 @@ def main():
     e2e_ms = r["e2e_ms"]
     from paper_2001_00138_b200 import replicas
     ms, e2e_ms = replicas.max_over_ranks([ms, e2e_ms], device="cuda")     # the slowest replica sets the time
-    conv_us = sum(r["layer_us"])
     roof_us = sum(c[2] for c in r["costs"])
-    achieved = r["flops"] / (conv_us * 1e-6) / 1e12
-    # dominant kernel: the tensor-core implicit GEMM (layers the planner gave to it)
-    tc = [(executed_tensor_flops(L, p), u) for L, p, u in zip(r["layer_objs"], r["plans"], r["layer_us"])]
-    tc_flops = sum(f for f, _ in tc)
-    tc_us = sum(u for f, u in tc if f > 0)
-    tc_peak = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0)))
-    tc_ach = tc_flops / (tc_us * 1e-6) / 1e12 if tc_us > 0 else 0.0
+    bytes_step = sum(c[1] for c in r["costs"])
+    achieved = r["flops"] / (ms * 1e-3) / 1e12                            # kept-weight TFLOP/s of the timed step
+    n_alu = sum(1 for c in r["costs"] if c[3] == "alu")
+
+    def tensor_pipe(res, step_ms):
+        """Executed 16-bit MMA flops of the tensor-core layers over their time INSIDE the chained step."""
+        tc = [(executed_tensor_flops(L, p), u) for L, p, u in zip(res["layer_objs"], res["plans"], res["in_step_us"])]
+        fl = sum(f for f, _ in tc)
+        us = sum(u for f, u in tc if f > 0)
+        capped = "sw_power_cap" in (res["clocks"].get("reasons") or [])
+        burst = float(peaks.get("bf16_tflops", 1590.0))
+        sustained = float(peaks.get("bf16_tflops_sustained", burst))
+        peak = sustained if capped else burst
+        ach = fl / (us * 1e-6) / 1e12 if us > 0 else 0.0
+        return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                "peak_source": f"{peak_kind} bf16 cuBLAS peak, " + ("sustained figure: the power cap was active during the timed region"
+                                                                   if capped else "burst figure: the timed region is short and ran at "
+                                                                   "full clocks with no power cap"),
+                "executed_flops_per_step": fl, "us_per_step": us, "launches_per_step": sum(1 for f, _ in tc if f > 0),
+                "step_us": step_ms * 1e3,
+                "what": "tcgen05 implicit GEMM kernels (bf16 hi/lo split, three products per fp32 product, zero-padded "
+                        "dense work): executed MMA flops / summed in-step time of the tensor-core layers, measured with "
+                        "events between the layers of the chained stack (patdnn_stack_run_timed)"}
+
     line = {
         "metric": "effective GFLOP/s on nonzero MACs, pattern-sparse 3x3 conv",
         "value": replicas.whole_job_value(r["flops"], ms * 1e-3, world) / 1e9,
@@ -611,46 +693,47 @@ def main():
                        "every step, two steps in flight (copies of one step overlap the kernels of the other); "
                        "blocking_ms_per_step = the same through patdnn_stack_run_host, one step at a time"},
         "gpu_launches": int(r["launches"]), "graph_ms_per_step": r["graph_ms_per_step"],
-        "roofline": {"bound": "tensor", "achieved": tc_ach, "peak": tc_peak, "unit": "TFLOP/s",
-                     "frac": tc_ach / tc_peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
-                     "frac_of_burst_peak": tc_ach / float(peaks.get("bf16_tflops", tc_peak)),
-                     "peak_source": f"{peak_kind} bf16 cuBLAS peak (sustained, kernel timed inside a long step)",
-                     "kernel": "conv_umma_halo_kernel / conv_umma_kernel (tcgen05 implicit GEMM, bf16 hi/lo split, three "
-                               "products per fp32 product); achieved = executed 16-bit MMA flops / summed launch time of "
-                               "the tensor-core layers (layout kernels included)",
-                     "launches_per_step": sum(1 for f, _ in tc if f > 0), "us_per_step": tc_us},
-        "north_star_roofline": {"definition": "per layer max(2*nonzero MACs / FP32 CUDA-core peak, algorithmic bytes / "
-                                              "measured HBM bandwidth); stack fraction = sum roofline / sum conv time",
-                                "bound": "alu", "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
-                                "peak_source": "148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
-                                "frac": achieved / ALU_PEAK_TFLOPS, "stack_roofline_us": roof_us,
-                                "stack_conv_us": conv_us, "stack_frac": roof_us / conv_us,
-                                "stack_frac_step": roof_us / (ms * 1e3),
-                                "note": "stack_frac uses the sum of per-layer launch times (each layer run alone, NCHW in "
-                                        "and out); stack_frac_step uses the timed step of the chained stack, pools included",
-                                "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
-        "layers": [{"name": n, "us": round(u, 2), "roofline_us": round(c[2], 2), "bound": c[3],
-                    "frac": round(c[2] / u, 3),
+        # The roofline of the metric: kept-weight flops at the FP32 CUDA-core peak against algorithmic bytes at the
+        # measured HBM bandwidth, per layer the slower of the two, summed over the step and divided by the step time.
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                     "frac": roof_us / (ms * 1e3), "traffic": TRAFFIC_BYTES_PER_LAUNCH, "traffic_note": TRAFFIC_NOTE,
+                     "definition": "per layer max(2 * nonzero MACs / FP32 CUDA-core peak, algorithmic bytes / measured HBM "
+                                   "bandwidth); frac = sum over the 13 layers / ms_per_step (whole chained step, fused pools "
+                                   "included); achieved = kept-weight flops of the step / ms_per_step",
+                     "peak_source": "derived: SMs x 128 FP32 lanes x 2 flop x max SM clock (an FFMA-chain probe measured 71.6)",
+                     "frac_alu_only": achieved / ALU_PEAK_TFLOPS, "roofline_us_per_step": roof_us,
+                     "flops_per_step": r["flops"], "algorithmic_bytes_per_step": bytes_step,
+                     "layers_alu_bound": n_alu, "layers_hbm_bound": 13 - n_alu,
+                     "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind},
+        "tensor_pipe": tensor_pipe(r, ms),
+        "layers": [{"name": n, "in_step_us": round(iu, 2), "standalone_us": round(u, 2), "roofline_us": round(c[2], 2),
+                    "bound": c[3], "frac_in_step": round(c[2] / iu, 3) if iu > 0 else None, "frac_standalone": round(c[2] / u, 3),
                     "kernel": "generated_fp32" if p.get("generated") else {3: "tiled", 4: "dense_tc"}.get(p["variant"], "generic"),
                     "tile": f"{p['tile_rows']}x{p['tile_cols']}x{p['filters_per_warp']}f", "grid": p["grid_x"]}
-                   for n, u, c, p in zip(r["names"], r["layer_us"], r["costs"], r["plans"])],
+                   for n, u, iu, c, p in zip(r["names"], r["layer_us"], r["in_step_us"], r["costs"], r["plans"])],
+        "layers_note": "in_step_us: the layer's kernels inside the chained step (events between layers); standalone_us: "
+                       "the layer called alone through patdnn_conv, NCHW in and out (layout kernel included)",
     }
     if rank == 0 and world == 1 and not args.no_extras:
         r1 = bench_stack(1, max(args.steps, 20), args.warmup, flush_l2=True)
-        conv1 = sum(r1["layer_us"])
         roof1 = sum(c[2] for c in r1["costs"])
         line["batch1"] = {"workload": "vgg16_3x3_stack_n1", "ms_per_step": r1["ms_per_step"],
                           "graph_ms_per_step": r1["graph_ms_per_step"],
-                          "stack_frac_graph": roof1 / (r1["graph_ms_per_step"] * 1e3),
                           "value": r1["flops"] / (r1["ms_per_step"] * 1e-3) / 1e9, "unit": "GFLOP/s",
-                          "l2": "256 MB buffer written between timed steps", "stack_conv_us": conv1,
-                          "stack_roofline_us": roof1, "stack_frac": roof1 / conv1,
-                          "stack_frac_step": roof1 / (r1["ms_per_step"] * 1e3),
-                          "layer_us": [round(u, 2) for u in r1["layer_us"]],
-                          "e2e_ms": r1["e2e_ms"]}
+                          "l2": "256 MB buffer written between timed steps",
+                          "roofline": {"bound": "alu", "achieved": r1["flops"] / (r1["ms_per_step"] * 1e-3) / 1e12,
+                                       "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                                       "frac": roof1 / (r1["ms_per_step"] * 1e3),
+                                       "frac_graph_replay": roof1 / (r1["graph_ms_per_step"] * 1e3),
+                                       "roofline_us_per_step": roof1},
+                          "tensor_pipe": tensor_pipe(r1, r1["ms_per_step"]),
+                          "in_step_us": [round(u, 2) for u in r1["in_step_us"]],
+                          "standalone_us": [round(u, 2) for u in r1["layer_us"]],
+                          "e2e_ms": r1["e2e_ms"], "gpu_launches": int(r1["launches"])}
         import oracle
         oracle.build()
         line["cpu_baseline"] = time_oracle_sample(synth)
+        line["parity"] = parity_against_oracle(synth, {args.batch: r["kept_out"], 1: r1["kept_out"]})
     elif rank == 0:
         line["cpu_baseline"] = None
     if rank == 0:

@@ -239,11 +239,17 @@ PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
  *                         in_host must stay untouched until the kernels of its batch ran, i.e. until its wait;
  *                         pinned host memory is needed for the copies to overlap.  All submits of a stack must use
  *                         the same stream.
+ *   patdnn_stack_run_timed  patdnn_stack_run with a CUDA event recorded on `stream` in front of every layer's launches
+ *                         and one behind the last; waits for the stack and writes the elapsed milliseconds of each
+ *                         layer (its kernels as launched inside the stack) to layer_ms, HOST [n].  For reports; the
+ *                         events between the launches switch off their overlap, so time whole steps with
+ *                         patdnn_stack_run
  *   patdnn_stack_out_shape  N, F, H, W of the stack's output
  * Errors: E_NULL, E_STACK, E_CUDA, E_NO_DEVICE.
  */
 PATDNN_API int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after, int32_t n, patdnn_stack *out);
 PATDNN_API int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream);
+PATDNN_API int patdnn_stack_run_timed(patdnn_stack s, const void *in, void *out, void *stream, float *layer_ms);
 PATDNN_API int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
 PATDNN_API int patdnn_stack_submit_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
 PATDNN_API int patdnn_stack_wait_host(patdnn_stack s);

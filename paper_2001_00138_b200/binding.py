@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "patdnn_encode", "patdnn_conv", "patdnn_conv_static", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
     "patdnn_stack_free", "patdnn_stack_submit_host", "patdnn_stack_wait_host", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
-    "patdnn_last_cuda_error", "patdnn_version", "patdnn_debug_wait",
+    "patdnn_last_cuda_error", "patdnn_version", "patdnn_debug_wait", "patdnn_stack_run_timed",
 )
 
 
@@ -86,6 +86,7 @@ def load() -> ctypes.CDLL:
     lib.patdnn_stack_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(i32), i32, ctypes.POINTER(vp)]
     lib.patdnn_stack_run.argtypes = [vp, vp, vp, vp]
     lib.patdnn_stack_run_host.argtypes = [vp, vp, vp, vp]
+    lib.patdnn_stack_run_timed.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float)]
     lib.patdnn_stack_submit_host.argtypes = [vp, vp, vp, vp]
     lib.patdnn_stack_wait_host.argtypes = [vp]
     lib.patdnn_stack_out_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 4
@@ -249,6 +250,13 @@ class Stack:
 
     def run(self, x, out, stream: int = 0) -> None:
         _check(load().patdnn_stack_run(self._h, _ptr(x), _ptr(out), stream), "patdnn_stack_run")
+
+    def run_timed(self, x, out, stream: int = 0) -> np.ndarray:
+        """patdnn_stack_run_timed: one synchronous pass; returns the milliseconds each layer took inside the stack."""
+        ms = np.zeros(len(self._layers), dtype=np.float32)
+        _check(load().patdnn_stack_run_timed(self._h, _ptr(x), _ptr(out), stream,
+                                             ms.ctypes.data_as(ctypes.POINTER(ctypes.c_float))), "patdnn_stack_run_timed")
+        return ms
 
     def run_host(self, x: np.ndarray, out: np.ndarray, stream: int = 0) -> None:
         assert x.flags.c_contiguous and out.flags.c_contiguous

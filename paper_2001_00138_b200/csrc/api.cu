@@ -558,7 +558,33 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
 // the second one's input directly (bias + ReLU applied, channels innermost, operands split): no tensor in NCHW form and
 // no layout kernel in between.  A pool between them is taken in the first one's epilogue where its shape allows a
 // poolable plan, else folded into the layout kernel of the second.
+static int stack_run_impl(patdnn_stack s, const void *in, void *out, void *stream, cudaEvent_t *ev);
+
 int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
+    return stack_run_impl(s, in, out, stream, nullptr);
+}
+
+int patdnn_stack_run_timed(patdnn_stack s, const void *in, void *out, void *stream, float *layer_ms) {
+    if (!s || !layer_ms) return PATDNN_E_NULL;
+    const int n = static_cast<int>(s->layers.size());
+    std::vector<cudaEvent_t> ev(n + 1, nullptr);
+    int rc = PATDNN_OK;
+    for (int i = 0; i <= n && !rc; ++i)
+        if (cudaEventCreate(&ev[i]) != cudaSuccess) rc = cuda_fail(cudaGetLastError(), "cudaEventCreate");
+    if (!rc) rc = stack_run_impl(s, in, out, stream, ev.data());
+    if (!rc) {
+        cudaError_t e = cudaEventSynchronize(ev[n]);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
+    }
+    for (int i = 0; i < n && !rc; ++i)
+        if (cudaEventElapsedTime(&layer_ms[i], ev[i], ev[i + 1]) != cudaSuccess) rc = cuda_fail(cudaGetLastError(), "cudaEventElapsedTime");
+    for (cudaEvent_t e : ev)
+        if (e) cudaEventDestroy(e);
+    return rc;
+}
+
+// ev (optional, n + 1 events): ev[i] is recorded in front of layer i's launches, ev[n] behind the last launch.
+static int stack_run_impl(patdnn_stack s, const void *in, void *out, void *stream, cudaEvent_t *ev) {
     if (!s || !in || !out) return PATDNN_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n = static_cast<int>(s->layers.size());
@@ -570,7 +596,11 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
     for (int i = 0; i < n; ++i) {
         patdnn_layer *h = s->layers[i];
         const patdnn_desc &d = h->desc;
-        if (d.N == 0) return PATDNN_OK;
+        if (d.N == 0) {
+            if (ev) for (int j = i; j <= n; ++j) CU(cudaEventRecord(ev[j], st));
+            return PATDNN_OK;
+        }
+        if (ev) CU(cudaEventRecord(ev[i], st));
         const bool last = (i == n - 1);
         const bool is_dense = h->variant == PATDNN_VARIANT_DENSE_TC;
         if (is_dense) {
@@ -635,8 +665,10 @@ int patdnn_stack_run(patdnn_stack s, const void *in, void *out, void *stream) {
     }
     if (cur_pool) {
         const patdnn_desc &ld = s->layers[n - 1]->desc;
-        return patdnn_maxpool2x2(cur, out, ld.N, ld.F, ld.H, ld.W, ld.dtype, stream);
+        const int rc = patdnn_maxpool2x2(cur, out, ld.N, ld.F, ld.H, ld.W, ld.dtype, stream);
+        if (rc) return rc;
     }
+    if (ev) CU(cudaEventRecord(ev[n], st));
     return PATDNN_OK;
 }
 

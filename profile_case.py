@@ -1,9 +1,11 @@
 """Runs one synthetic layer a few times through the C ABI -- the small case to put under ``ncu``.
 
-    python -m paper_2001_00138_b200.profile_case --layer vgg6 --batch 4 --reps 3 [--variant tiled]
+    python profile_case.py --layer vgg6 --batch 4 --reps 3 [--variant tiled]
 
 Layers: ``cfg1``, ``cfg2``, ``vggK`` (K = 1..13, VGG-16-shaped layer K), ``resnetK`` (K = 1..4, fp16),
-``sweep:P:PRUNE`` (512->512 @14x14), ``custom:F:C:H:W:P:PRUNE``.  Prints the mean launch time measured with CUDA events.
+``sweep:P:PRUNE`` (512->512 @14x14), ``custom:F:C:H:W:P:PRUNE``.  ``--chain M`` (vggK only) runs layers K .. K+M-1 as a
+stack, so that the in-stack kernels (first layer writing the next layer's operands, fused pools) can be captured.
+Prints the mean launch time measured with CUDA events.
 """
 from __future__ import annotations
 
@@ -11,7 +13,7 @@ import argparse
 import os
 import sys
 
-sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 
 
 def make(layer: str, batch: int):
@@ -34,16 +36,43 @@ def make(layer: str, batch: int):
     raise SystemExit(f"unknown layer {layer}")
 
 
+def run_chain(args, torch, B):
+    from paper_2001_00138_b200 import synth
+    first = int(args.layer[3:]) - 1
+    idx = list(range(first, first + args.chain))
+    layers = [synth.vgg16_layer(i, N=args.batch) for i in idx]
+    handles = [B.encode(L.weights, L.mask, L.patterns, N=args.batch, H=L.H, W=L.W, relu=True, bias=L.bias) for L in layers]
+    stack = B.Stack(handles, [1 if i in synth.VGG16_POOL_AFTER else 0 for i in idx])
+    L0 = layers[0]
+    x = torch.rand((args.batch, L0.C, L0.H, L0.W), device="cuda")
+    y = torch.empty(stack.out_shape(), device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    stack.run(x, y, st)
+    torch.cuda.synchronize()
+    tot = None
+    for _ in range(args.reps):
+        ms = stack.run_timed(x, y, st)
+        tot = ms if tot is None else tot + ms
+    print(f"stack of {[L.name for L in layers]} N={args.batch}: per-layer us {[round(float(v) * 1e3 / args.reps, 1) for v in tot]}")
+    stack.free()
+    for h in handles:
+        h.free()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--layer", default="vgg6")
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--variant", default="auto", choices=["auto", "noopt", "reorder", "tiled", "dense"])
+    ap.add_argument("--chain", type=int, default=1)
     args = ap.parse_args()
     import torch
     from paper_2001_00138_b200 import binding as B, build
     build.build_library()
+    if args.chain > 1:
+        run_chain(args, torch, B)
+        return
     L = make(args.layer, args.batch)
     N = L.N if args.layer in ("cfg1", "cfg2") else args.batch
     dt = B.F16 if L.dtype == "f16" else B.F32
