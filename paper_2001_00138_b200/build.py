@@ -8,9 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatdnn.so")
-SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "smallc_split.cu", "smallc_jit.cu", "tiled_inst_4x8.cu",
+SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "umma_chain.cu", "smallc_split.cu", "smallc_jit.cu", "tiled_inst_4x8.cu",
            "tiled_inst_4x4.cu", "tiled_inst_2x8.cu", "fkw_encoder.cpp", "tiled_plan.cpp"]
-HEADERS = ["kernels.hpp", "kernels_tiled.cuh", "fkw_encoder.hpp", os.path.join("generated", "tiled_cases.inc"),
+HEADERS = ["kernels.hpp", "umma_ptx.cuh", "kernels_tiled.cuh", "fkw_encoder.hpp", os.path.join("generated", "tiled_cases.inc"),
            os.path.join("..", "..", "include", "patdnn.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--threads", "0"]

@@ -80,6 +80,7 @@ struct patdnn_layer {
     int dense_pool_state = 0;                // 0 = not tried, 1 = ready, -1 = this layer's shape has no such plan
     // staging buffers of patdnn_conv_host
     void *d_in_stage = nullptr, *d_out_stage = nullptr;
+    unsigned long long *chain_bar = nullptr;           // grid-barrier words of a stack's chained launch that reports to this handle's status
 };
 
 struct patdnn_stack_s {
@@ -93,6 +94,15 @@ struct patdnn_stack_s {
     std::vector<int> smallc;                  // per layer: index into smallc_w, or -1
     std::vector<SmallCWeights> smallc_w;      // few-channel layers fused with the layout of the tensor-core layer after them
     std::vector<SmallCJit *> smallc_jit;      // the same layers as run-time generated code (nullptr: static kernel)
+    // runs of small tensor-core layers executed by one persistent cooperative kernel
+    struct ChainRun {
+        int first = 0, count = 0, grid = 0;
+        ChainParams params{};
+    };
+    std::vector<ChainRun> chains;
+    std::vector<int> chain_at;                // per layer: index into chains of the run that starts here, or -1
+    float *d_partial = nullptr;               // partial-tile scratch shared by the runs
+    unsigned long long *d_bar = nullptr;      // grid-barrier arrival counter
     void *buf[2] = {nullptr, nullptr};
     void *d_in = nullptr, *d_out = nullptr;   // staging buffers of patdnn_stack_run_host
     size_t buf_bytes = 0, in_bytes = 0, out_bytes = 0;
@@ -406,6 +416,7 @@ int patdnn_check(patdnn_handle h) {
         CU(cudaMemcpy(&st, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
         if (st != 0) {
             cudaMemset(h->d_status, 0, sizeof(int));
+            if (h->chain_bar) cudaMemset(h->chain_bar, 0, 16);   // the grid barrier may have been left half-way
             return PATDNN_E_DEVICE_TIMEOUT;
         }
     }
@@ -541,6 +552,73 @@ int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after,
         s->smallc_jit.push_back(smallc_jit_build(h->fkw, h->bias, d.C, d.relu, d.dtype == PATDNN_F16, nullptr));
         s->smallc[i] = static_cast<int>(s->smallc_w.size()) - 1;
     }
+    // Runs of consecutive tensor-core layers with at most one tile per SM (small batches) as one persistent kernel per
+    // run.  Opt-in (PATDNN_DEBUG=chain=1): correct, but measured no faster than one kernel per layer -- VGG-shaped stack
+    // at batch 1: 205 us against 200 us; its layers are bound by the L2 -> SM traffic of their operand tiles (about
+    // 14 TB/s in both forms), and the exchange of partial tiles through global memory with two grid barriers costs as
+    // much per layer (about 8 us) as the launch, set-up and cluster exchange it replaces.
+    s->chain_at.assign(n, -1);
+    const int cgrid = debug_option("chain", 0) == 1 ? chain_grid(dtype) : 0;
+    if (cgrid > 0) {
+        auto eligible = [&](int i, ChainLayer &L) {
+            patdnn_layer *h = s->layers[i];
+            const patdnn_desc &d = h->desc;
+            if (h->variant != PATDNN_VARIANT_DENSE_TC || h->dense.im2col || h->dense.gather || h->dense.taps != 9 || d.N < 1) return false;
+            L = ChainLayer();
+            if (!chain_box(d.N, d.H, d.W, s->pool[i] != 0, L)) return false;
+            L.N = d.N; L.C = d.C; L.H = d.H; L.W = d.W; L.F = d.F;
+            L.n_ftiles = (d.F + 127) / 128;
+            L.KB = h->dense.KB; L.ipt = 9 * L.KB;
+            L.n_tiles = L.tiles_x * L.tiles_y * L.tiles_n * L.n_ftiles;
+            L.total = L.n_tiles * L.ipt;
+            L.gw = std::min(cgrid, L.total);
+            if (static_cast<long long>(L.total) * cgrid >= (1ll << 31)) return false;
+            L.box_bytes = L.TW * L.TH * L.TN * 128;
+            L.relu = d.relu; L.pool = s->pool[i] != 0;
+            L.bias = h->d_bias;
+            return L.n_tiles <= cgrid;                            // a chunk then touches at most two tiles
+        };
+        int i = 0;
+        while (i < n) {
+            ChainLayer L;
+            if (!eligible(i, L)) { ++i; continue; }
+            patdnn_stack_s::ChainRun run;
+            run.first = i; run.grid = cgrid;
+            bool good = true;
+            while (i < n && run.count < kChainMaxLayers && eligible(i, L)) {
+                patdnn_layer *h = s->layers[i];
+                const bool more = i + 1 < n && run.count + 1 < kChainMaxLayers;
+                ChainLayer nextL;
+                const bool next_in = more && eligible(i + 1, nextL);
+                const bool next_dense = i + 1 < n && s->layers[i + 1]->variant == PATDNN_VARIANT_DENSE_TC && !s->layers[i + 1]->dense.im2col;
+                if (next_in || next_dense) { L.out_mode = 3; L.out = s->layers[i + 1]->d_act; L.out_cp = s->layers[i + 1]->dense.Cp; }
+                else { L.out_mode = 0; L.out = nullptr; L.out_cp = 0; }          // NCHW destination patched in at run time
+                if (make_chain_maps(run.params.mapA[run.count], run.params.mapB[run.count], L, h->dense, h->d_act, h->d_wdense, dtype) != PATDNN_OK) {
+                    good = false;
+                    break;
+                }
+                run.params.layer[run.count++] = L;
+                ++i;
+            }
+            if (!good || run.count < 2) { if (run.count == 0) ++i; continue; }   // single layers stay on their own kernels
+            run.params.n_layers = run.count;
+            run.params.stages = chain_stages(dtype);
+            run.params.status = s->layers[run.first]->d_status;
+            s->chain_at[run.first] = static_cast<int>(s->chains.size());
+            s->chains.push_back(run);
+        }
+        if (!s->chains.empty()) {
+            cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&s->d_partial), chain_partial_bytes(cgrid));
+            if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&s->d_bar), 16);
+            if (e == cudaSuccess) e = cudaMemset(s->d_bar, 0, 16);
+            if (e != cudaSuccess) { patdnn_stack_free(s); return cuda_fail(e, "cudaMalloc(chain scratch)"); }
+            for (auto &run : s->chains) {
+                run.params.partial = s->d_partial;
+                run.params.bar = s->d_bar;
+                s->layers[run.first]->chain_bar = s->d_bar;
+            }
+        }
+    }
     s->oN = N; s->oF = C; s->oH = H; s->oW = W;
     s->buf_bytes = std::max<size_t>(max_bytes, 16);
     const patdnn_desc &d0 = handles[0]->desc;
@@ -624,6 +702,29 @@ static int stack_run_impl(patdnn_stack s, const void *in, void *out, void *strea
                                                   curH, curW, h->dense.Cp, h->dense.S, st);
                 if (e != cudaSuccess) return cuda_fail(e, "layout kernel launch");
                 g_launches.fetch_add(1, std::memory_order_relaxed);
+            }
+            if (s->chain_at[i] >= 0) {
+                // this layer's operands are in place: one persistent kernel runs it and the layers chained behind it
+                const patdnn_stack_s::ChainRun &run = s->chains[s->chain_at[i]];
+                const int e_idx = run.first + run.count - 1;
+                ChainParams cp = run.params;
+                cp.spin_limit = h->spin_limit; cp.test_skip_load = h->test_skip_load;
+                const patdnn_desc &ld = s->layers[e_idx]->desc;
+                if (cp.layer[run.count - 1].out_mode == 0) {
+                    void *dst = (e_idx == n - 1) ? out : s->buf[which];
+                    cp.layer[run.count - 1].out = dst;
+                    cur = dst; which ^= 1; direct = false;
+                } else {
+                    direct = true;
+                }
+                if (ev) for (int j = i + 1; j <= e_idx; ++j) CU(cudaEventRecord(ev[j], st));
+                cudaError_t ce = chain_launch(cp, run.grid, d.dtype, st);
+                if (ce != cudaSuccess) return cuda_fail(ce, "chained tensor-core kernel launch");
+                g_launches.fetch_add(1, std::memory_order_relaxed);
+                cur_pool = false;                                 // pools inside and behind the run are taken while reducing
+                curH = s->pool[e_idx] ? ld.H / 2 : ld.H; curW = s->pool[e_idx] ? ld.W / 2 : ld.W;
+                i = e_idx;
+                continue;
             }
             patdnn_layer *next = (next_dense && (!s->pool[i] || fuse_pool)) ? s->layers[i + 1] : nullptr;
             void *dst = next ? nullptr : ((last && !s->pool[i]) ? out : s->buf[which]);
@@ -746,6 +847,10 @@ int patdnn_stack_free(patdnn_stack s) {
         if (s->ev_out[b]) cudaEventDestroy(s->ev_out[b]);
     }
     for (SmallCJit *j : s->smallc_jit) smallc_jit_free(j);
+    if (s->d_partial) cudaFree(s->d_partial);
+    if (s->d_bar) cudaFree(s->d_bar);
+    for (patdnn_layer *h : s->layers)
+        if (h && h->chain_bar == s->d_bar) h->chain_bar = nullptr;
     if (s->h2d) cudaStreamDestroy(s->h2d);
     if (s->d2h) cudaStreamDestroy(s->d2h);
     delete s;

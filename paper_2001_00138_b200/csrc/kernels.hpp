@@ -203,6 +203,39 @@ SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int 
 cudaError_t smallc_jit_launch(SmallCJit *j, const void *in, void *dst, int N, int H, int W, cudaStream_t st);
 void smallc_jit_free(SmallCJit *j);
 
+// ---- several tensor-core layers in one persistent cooperative kernel (umma_chain.cu) -----------------------------------
+constexpr int kChainMaxLayers = 12;
+struct ChainLayer {
+    int N, C, H, W, F;
+    int TW, TH, TN, tiles_x, tiles_y, tiles_n, n_ftiles;   // pixel box, boxes per image axis / batch, filter tiles of 128
+    int KB, ipt;                // channel blocks of 64; iterations per tile = 9 * KB
+    int n_tiles, total;         // tiles of the layer; total = n_tiles * ipt, cut into equal chunks over the working CTAs
+    int gw;                     // working CTAs of this layer = min(grid, total)
+    int box_bytes;              // TW * TH * TN * 128
+    int relu, pool;             // pool: 2x2 max-pool taken while reducing
+    int out_mode, out_cp;       // 0: NCHW tensor of the layer's dtype; 3: the next layer's split operands [S][N][h][w][out_cp]
+    const float *bias;          // DEVICE [F]
+    void *out;
+};
+struct ChainParams {
+    CUtensorMap mapA[kChainMaxLayers], mapB[kChainMaxLayers];
+    ChainLayer layer[kChainMaxLayers];
+    int n_layers, stages;
+    float *partial;             // DEVICE scratch: 2 * CTAs slots of 128 x 128 fp32; CTA c's partial of tile t is slot c + t
+    unsigned long long *bar;    // DEVICE: arrivals at the grid barrier; only grows, a multiple of the grid size between launches
+    int *status;                // DEVICE word: 0 = ok, else the role whose bounded wait expired
+    uint32_t spin_limit;        // polls per bounded wait (0 = default)
+    int test_skip_load;         // test hook: producers leave out the activation loads of this (1-based) iteration of their
+                                // first layer's chunk, so that a bounded wait runs out (0 = off)
+};
+bool chain_box(int N, int H, int W, bool pool, ChainLayer &L);
+int chain_stages(int dtype);
+size_t chain_partial_bytes(int grid);
+int chain_grid(int dtype);                                 // CTAs of the cooperative launch (0: not available here)
+cudaError_t chain_launch(const ChainParams &p, int grid, int dtype, cudaStream_t st);
+// tensor maps of one chained layer over its split activations and dense weights (PATDNN_* status)
+int make_chain_maps(CUtensorMap &mapA, CUtensorMap &mapB, const ChainLayer &L, const DensePlan &pl, void *d_act, void *d_w, int dtype);
+
 bool dense_supported(int F, int C, int N, int H, int W);
 // pool_tiles: only pixel boxes whose epilogue can max-pool in registers (one image per box, 2/4/8/16 pixels wide, starting
 // on even rows); sets pl.poolable.  force_bn pins the filter tile width, so that a second plan of a layer shares the

@@ -36,6 +36,7 @@
 
 #include "../../include/patdnn.h"
 #include "kernels.hpp"
+#include "umma_ptx.cuh"
 
 namespace patdnn {
 
@@ -45,92 +46,6 @@ namespace {
 constexpr int kThreads = 320;                // general kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kHaloThreads = 320;            // persistent kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kGatherThreads = 256;          // plus eight gather warps for layers whose operand rows are built in the kernel
-constexpr int kTileM = 128;
-constexpr int kKBlock = 64;                  // channels per stage: 64 x 2 bytes = one 128-byte swizzle row
-constexpr uint32_t kSpinLimit = 1u << 21;    // default bound of mbarrier polling: each poll may block up to ~1 us (hint below)
-
-// Where a bounded wait reports to and how many polls it may take (DenseParams::spin_limit, 0 = the default).
-struct WaitCtx {
-    int *word;
-    uint32_t limit;
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait: returns false (and leaves *status set) when the phase did not complete within the polling budget.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &status, int code) {
-    for (uint32_t i = 0; i < status.limit; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred P1;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2, 0x400;\n\t"
-            "selp.b32 %0, 1, 0, P1;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-        // another role already gave up?  (a global read: only now and then, it would otherwise sit on every wake-up path)
-        if ((i & 15u) == 15u && *reinterpret_cast<volatile int *>(status.word) != 0) return false;
-    }
-    atomicCAS(status.word, 0, code);
-    return false;
-}
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// K-major, 128-byte-swizzled shared-memory matrix descriptor: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);            // start address, 16-byte units
-    d |= static_cast<uint64_t>(1) << 16;                            // leading byte offset (unused for swizzled K-major)
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;                    // stride byte offset between 8-row groups
-    d |= static_cast<uint64_t>(1) << 46;                            // descriptor version for sm_100
-    d |= static_cast<uint64_t>(2) << 61;                            // layout: 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: fp32 accumulate, A and B both K-major in the same 16-bit format (0 = f16, 1 = bf16).
-__host__ __device__ constexpr uint32_t instr_desc(int fmt, int n) {
-    return (1u << 4) | (static_cast<uint32_t>(fmt) << 7) | (static_cast<uint32_t>(fmt) << 10) |
-           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
-}
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(addr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 // ---- transition into a tensor-core layer: finish the producer, change layout, split operands ---------------------
 // src is NCHW with Hs x Ws pixels: the caller's input (float or half), or the raw fp32 sums of the previous
 // tensor-core layer, in which case that layer's bias + ReLU are applied here and (clear) the sums are zeroed after
@@ -1535,6 +1450,33 @@ int make_dense_maps(DensePlan &pl, void *d_act, void *d_w, int N, int H, int W, 
         cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)pl.BN, 1, 1};
         cuuint32_t es[4] = {1, 1, 1, 1};
         if (enc(&pl.mapB, dt, 4, d_w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    return PATDNN_OK;
+}
+
+int make_chain_maps(CUtensorMap &mapA, CUtensorMap &mapB, const ChainLayer &L, const DensePlan &pl, void *d_act, void *d_w, int dtype) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return PATDNN_E_CUDA;
+    const CUtensorMapDataType dt = dtype == PATDNN_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    {
+        cuuint64_t dims[5] = {(cuuint64_t)pl.Cp, (cuuint64_t)L.W, (cuuint64_t)L.H, (cuuint64_t)L.N, (cuuint64_t)pl.S};
+        cuuint64_t strides[4] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)L.W * pl.Cp * 2, (cuuint64_t)L.H * L.W * pl.Cp * 2,
+                                 (cuuint64_t)L.N * L.H * L.W * pl.Cp * 2};
+        cuuint32_t box[5] = {(cuuint32_t)kKBlock, (cuuint32_t)L.TW, (cuuint32_t)L.TH, (cuuint32_t)L.TN, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (enc(&mapA, dt, 5, d_act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PATDNN_E_CUDA;
+    }
+    {
+        // filter tiles of 128 whatever tile width the handle's weight image was padded for: rows past Fp read as zero
+        cuuint64_t dims[4] = {(cuuint64_t)pl.Cp, (cuuint64_t)pl.Fp, (cuuint64_t)pl.taps, (cuuint64_t)pl.S};
+        cuuint64_t strides[3] = {(cuuint64_t)pl.Cp * 2, (cuuint64_t)pl.Fp * pl.Cp * 2, (cuuint64_t)pl.taps * pl.Fp * pl.Cp * 2};
+        cuuint32_t box[4] = {(cuuint32_t)kKBlock, 128u, 1, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        if (enc(&mapB, dt, 4, d_w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return PATDNN_E_CUDA;
     }

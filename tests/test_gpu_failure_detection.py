@@ -48,3 +48,48 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_keeps_working(ks, monke
     layer.check()
     assert_close(out.cpu().numpy(), ref, TOL_F32, "after the expired wait")
     layer.free()
+
+
+def test_a_wait_that_runs_out_in_the_persistent_multi_layer_kernel(monkeypatch):
+    """The chained kernel has mbarrier waits AND a barrier over all its CTAs.  With one iteration's activation loads
+    withheld in every CTA, the MMA threads' waits run out, the status word stops every other wait and grid barrier,
+    the kernel returns, patdnn_check on the run's first handle reports the timeout (and clears the barrier words), and
+    the same stack then runs normally.  (The kernel is opt-in: PATDNN_DEBUG=chain=1.)"""
+    monkeypatch.setenv("PATDNN_DEBUG", "chain=1")
+    import oracle
+    import torch
+    build.build_library()
+    from paper_2001_00138_b200 import binding as B
+    N, H, W, chans = 1, 14, 14, [256, 256, 128, 192]
+    x = synth.make_layer("x", F=1, C=chans[0], N=N, H=H, W=W, seed=5, x_dist="normal").x
+    cur, handles = x, []
+    for i in range(3):
+        L = synth.make_layer(f"t{i}", F=chans[i + 1], C=chans[i], N=N, H=H, W=W, seed=700 + i, prune=0.5, bias_std=0.2,
+                             draw_input=False, w_std=float(np.sqrt(2.0 / (4 * chans[i] * 0.5))))
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=H, W=W, relu=True, bias=L.bias, variant=B.VARIANT_DENSE_TC))
+        cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+    stack = B.Stack(handles, [0, 0, 0])
+    st = torch.cuda.current_stream().cuda_stream
+    xt = torch.from_numpy(x).cuda()
+    out = torch.zeros(cur.shape, device="cuda")
+    B.reset_launch_count()
+    stack.run(xt, out, st)
+    handles[0].check()
+    assert B.launch_count() == 2, "layout kernel + one persistent kernel"
+    assert_close(out.cpu().numpy(), cur, TOL_F32 * 3 ** 0.5, "before the expired wait")
+
+    handles[0].debug_wait(1024, 1)                 # the first iteration's activation tile never arrives
+    stack.run(xt, out, st)
+    with pytest.raises(B.PatdnnError) as e:
+        handles[0].check()
+    assert e.value.status == E_DEVICE_TIMEOUT
+    handles[0].debug_wait(0, 0)
+    out.fill_(float("nan"))
+    stack.run(xt, out, st)
+    for h in handles:
+        h.check()
+    assert_close(out.cpu().numpy(), cur, TOL_F32 * 3 ** 0.5, "after the expired wait")
+    stack.free()
+    for h in handles:
+        h.free()
+

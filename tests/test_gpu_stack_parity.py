@@ -78,7 +78,8 @@ def test_every_benchmark_layer_in_its_in_stack_form(i, N):
     else:
         assert plan["variant"] == DENSE
         # no layout kernel and no pooling kernel behind the first layer: its GEMM (plus a K-split tail launch where
-        # the plan has one) and the identity's GEMM (ditto); the only layout kernel is the one in front of the stack
+        # the plan has one) and the identity's GEMM (ditto) -- or one persistent kernel for both at batch 1; the only
+        # layout kernel is the one in front of the stack
         assert launches <= 1 + 2 + 2
     assert_close(got, _oracle_one_layer(L, x, pool), TOL_F32, f"vgg L{i + 1} N={N} in-stack")
 
@@ -104,14 +105,20 @@ IN_STACK_CASES = [
 ]
 
 
+@pytest.mark.parametrize("chained", [True, False])
 @pytest.mark.parametrize("generated", [True, False])
 @pytest.mark.parametrize("case", IN_STACK_CASES)
-def test_in_stack_paths_at_the_single_layer_tolerance(case, generated, monkeypatch):
+def test_in_stack_paths_at_the_single_layer_tolerance(case, generated, chained, monkeypatch):
+    """chained = False: one kernel per layer, epilogues that write the successor's operands (the default);
+    chained = True: the stack may run consecutive small tensor-core layers as one persistent kernel (opt-in)."""
     N, C, F, H, W, pool, dtype, variant, prune = case
+    opts = ["chain=1"] if chained else []
     if not generated:
         if C > 4:
             pytest.skip("the run-time generated kernel only exists for few-channel first layers")
-        monkeypatch.setenv("PATDNN_DEBUG", "jit=0")
+        opts.append("jit=0")
+    if opts:
+        monkeypatch.setenv("PATDNN_DEBUG", ",".join(opts))
     L = synth.make_layer("in_stack", F=F, C=C, N=N, H=H, W=W, seed=1234 + C + F, prune=prune, bias_std=0.3,
                          x_dist="normal", dtype=dtype, w_std=float(np.sqrt(2.0 / (4 * C * (1 - prune)))))
     got, _, _ = _run_with_identity(L, L.x, pool, variant=variant, dtype=dtype)
@@ -154,3 +161,61 @@ def test_benchmark_stack_whole_images_against_the_chained_oracle(N):
     stack.free()
     for h in handles:
         h.free()
+
+
+# chains of tensor-core layers small enough for the persistent multi-layer kernel
+# (N, H, W, channels per layer boundary, pool flags, dtype)
+CHAIN_CASES = [
+    (1, 28, 28, [64, 128, 128, 256, 192], [0, 1, 0, 0], "f32"),
+    (1, 14, 14, [512, 512, 512, 512], [0, 0, 0], "f32"),
+    (2, 20, 24, [96, 130, 70, 64], [1, 0, 1], "f32"),          # ragged filter tiles and channel blocks, two pools
+    (3, 12, 16, [64, 64, 200, 40, 64, 96], [0, 1, 0, 0, 1], "f32"),
+    (1, 56, 56, [128, 256, 256], [0, 1], "f32"),                # 28 pixel tiles x 2 filter tiles per layer
+    (2, 14, 10, [64, 96, 128, 40], [0, 1, 0], "f16"),
+    (1, 24, 24, [64, 64, 64, 96, 40], [1, 1, 0, 0], "f16"),
+    (5, 9, 7, [70, 33, 129, 64], [0, 0, 0], "f32"),             # odd extents (no pool), several images per tile
+]
+
+
+@pytest.mark.parametrize("case", CHAIN_CASES)
+def test_chained_layers_in_one_persistent_kernel(case, monkeypatch):
+    """Runs of small tensor-core layers: after the layout kernel in front, the whole run is ONE launch; the result must
+    equal the chained oracle and the host-buffer call must give the same bits."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    monkeypatch.setenv("PATDNN_DEBUG", "chain=1")               # the persistent multi-layer kernel is opt-in
+    N, H, W, chans, pools, dtype = case
+    dt = B.F16 if dtype == "f16" else B.F32
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    tol = TOL_F16 if dtype == "f16" else TOL_F32
+    nl = len(chans) - 1
+    x = synth.make_layer("x", F=1, C=chans[0], N=N, H=H, W=W, seed=77, x_dist="normal", dtype=dtype).x
+    cur, handles, h, w = x.astype(np.float32), [], H, W
+    for i in range(nl):
+        L = synth.make_layer(f"ch{i}", F=chans[i + 1], C=chans[i], N=N, H=h, W=w, seed=600 + i, prune=0.5, bias_std=0.2,
+                             draw_input=False, dtype=dtype, w_std=float(np.sqrt(2.0 / (4 * chans[i] * 0.5))))
+        handles.append(B.encode(L.weights, L.mask, L.patterns, N=N, H=h, W=w, dtype=dt, relu=True, bias=L.bias, variant=DENSE))
+        cur = oracle.conv3x3(cur, L.weights, L.mask, L.bias, True)
+        if pools[i]:
+            cur = oracle.maxpool2x2(cur)
+            h, w = h // 2, w // 2
+        if dtype == "f16" and i < nl - 1:
+            cur = cur.astype(np.float16).astype(np.float32)       # the layer boundary stores fp16
+    stack = B.Stack(handles, pools)
+    assert stack.out_shape() == cur.shape
+    out = torch.full(cur.shape, float("nan"), device="cuda", dtype=tdt)
+    B.reset_launch_count()
+    stack.run(torch.from_numpy(x).to("cuda", dtype=tdt), out, torch.cuda.current_stream().cuda_stream)
+    for hd in handles:
+        hd.check()
+    assert B.launch_count() == 2, "one layout kernel, then one persistent kernel for the whole run"
+    got = out.float().cpu().numpy()
+    assert_close(got, cur, chain_tol(nl, tol), f"chained run {case}")
+    out_h = np.empty(cur.shape, dtype=np.float16 if dtype == "f16" else np.float32)
+    stack.run_host(np.ascontiguousarray(x.astype(out_h.dtype)), out_h)
+    assert np.array_equal(out_h.astype(np.float32), got)
+    stack.free()
+    for hd in handles:
+        hd.free()
+
