@@ -199,6 +199,60 @@ __global__ void __launch_bounds__(256) transition_vec_kernel(float *__restrict__
     }
 }
 
+// The same operation without pooling for ANY image size and both source types: a channel's H*W pixels are contiguous in
+// NCHW, so the image is treated as a flat [C][H*W] matrix and transposed in 64 x 64 tiles through shared memory --
+// loads run along the pixels (a warp reads 32 consecutive elements of one channel), stores along the channels (four
+// lanes write the 64 channels of one pixel, 32 bytes each per plane).  grid = (ceil(HW/64), Cp/64, N), block = 256.
+template <typename T>
+__global__ void __launch_bounds__(256) transition_flat_kernel(const T *__restrict__ src, uint16_t *__restrict__ dst, int N, int C,
+                                                              int HW, int Cp, int S) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float tile[64][65];                               // [channel][pixel]
+    const int p0 = blockIdx.x * 64, c0 = blockIdx.y * 64, n = blockIdx.z;
+    const int tid = threadIdx.x;
+    {
+        const int px = tid & 63, p = p0 + px;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int cc = 4 * k + (tid >> 6), c = c0 + cc;
+            float v = 0.f;
+            if (c < C && p < HW) {
+                const T raw = src[(static_cast<size_t>(n) * C + c) * HW + p];
+                if constexpr (sizeof(T) == 2) v = __half2float(raw); else v = raw;
+            }
+            tile[cc][px] = v;
+        }
+    }
+    __syncthreads();
+    const int px = tid >> 2, sub = tid & 3, p = p0 + px;
+    if (p >= HW) return;
+    uint32_t hi[8], lo[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float a = tile[16 * sub + 2 * j][px], b = tile[16 * sub + 2 * j + 1][px];
+        if (S == 2) {
+            const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+            const __nv_bfloat16 al = __float2bfloat16_rn(a - __bfloat162float(ah));
+            const __nv_bfloat16 bl = __float2bfloat16_rn(b - __bfloat162float(bh));
+            hi[j] = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
+            lo[j] = static_cast<uint32_t>(__bfloat16_as_ushort(al)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
+        } else {
+            hi[j] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(a))) |
+                    (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(b))) << 16);
+        }
+    }
+    const size_t o = (static_cast<size_t>(n) * HW + p) * Cp + c0 + 16 * sub;
+    uint4 *d0 = reinterpret_cast<uint4 *>(dst + o);
+    d0[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    d0[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+    if (S == 2) {
+        uint4 *d1 = reinterpret_cast<uint4 *>(dst + static_cast<size_t>(N) * HW * Cp + o);
+        d1[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        d1[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+    }
+}
+
 // Layers with very few input channels (9*C <= 64, e.g. an RGB first layer): gather the 3x3 neighbourhood into the
 // channel dimension, k = 9*c + tap, so that the whole layer is ONE 64-deep GEMM step instead of nine mostly-padding ones.
 // dst is [S][N][H][W][64].  A block stages the three input rows of a 32-pixel row segment for all channels in shared
@@ -1517,6 +1571,17 @@ cudaError_t launch_transition(const void *src, int src_is_half, void *dst, const
     const int H = pool ? Hs / 2 : Hs, W = pool ? Ws / 2 : Ws;
     if (N == 0 || H == 0 || W == 0) return cudaSuccess;
     const int gz = N * (Cp / 64);
+    // no pool, nothing to finish: the flat transpose, unless float4 rows are available (same traffic, fewer instructions)
+    if (!pool && !bias && !relu && !clear && N <= 65535 && Cp / 64 <= 65535 &&
+        (src_is_half || Ws % 4 != 0 || (reinterpret_cast<uintptr_t>(src) & 15) != 0)) {
+        const int HW = Hs * Ws;
+        dim3 grid((HW + 63) / 64, Cp / 64, N);
+        if (src_is_half)
+            return launch_pdl(transition_flat_kernel<__half>, grid, dim3(256), 0, st, 1, static_cast<const __half *>(src),
+                              static_cast<uint16_t *>(dst), N, C, HW, Cp, S);
+        return launch_pdl(transition_flat_kernel<float>, grid, dim3(256), 0, st, 1, static_cast<const float *>(src),
+                          static_cast<uint16_t *>(dst), N, C, HW, Cp, S);
+    }
     if (!src_is_half && Ws % 4 == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
         float *fs = static_cast<float *>(const_cast<void *>(src));
         uint16_t *d16 = static_cast<uint16_t *>(dst);
