@@ -462,19 +462,24 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     if (warp == 0) {
         if (lane == 0) {
             const uint32_t tx_bytes = S * (p.box_bytes + B_BYTES);
+            // ring slot, its use count and the (channel block, tap) of the iteration advance without divisions: this one
+            // thread's instruction stream is what a short channel/tap loop waits for
+            int s = 0, use = 0, cb = it0 / p.taps, tap = it0 - cb * p.taps;
+            const uint32_t smem_base = smem_u32(smem);
             for (int it = 0; it < iters; ++it) {
-                const int s = it % stages, use = it / stages;
                 if (use > 0 && !mbar_wait(bar_empty + 8 * s, (use - 1) & 1, status, 1)) break;
-                if (it + 1 == p.test_skip_load) continue;       // test hook: this iteration's loads never arrive
-                const int cb = (it0 + it) / p.taps, tap = (it0 + it) - cb * p.taps;
-                const int r = p.taps == 9 ? tap / 3 : 1, sx = p.taps == 9 ? tap - 3 * r : 1;
-                const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
-                if (it >= npre) mbar_expect_tx(bar_full + 8 * s, tx_bytes);   // the first slots were armed with their weights
+                if (it + 1 != p.test_skip_load) {                // test hook: that iteration's loads never arrive
+                    const int r = p.taps == 9 ? tap / 3 : 1, sx = p.taps == 9 ? tap - 3 * r : 1;
+                    const uint32_t base = smem_base + s * STAGE_BYTES;
+                    if (it >= npre) mbar_expect_tx(bar_full + 8 * s, tx_bytes);   // the first slots were armed with their weights
 #pragma unroll
-                for (int sp = 0; sp < S; ++sp) {
-                    tma_load_5d(base + sp * A_BYTES, &mapA, bar_full + 8 * s, cb * kKBlock, x0 + sx - 1, y0 + r - 1, n0, sp);
-                    if (it >= npre) tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * s, cb * kKBlock, f0, tap, sp);
+                    for (int sp = 0; sp < S; ++sp) {
+                        tma_load_5d(base + sp * A_BYTES, &mapA, bar_full + 8 * s, cb * kKBlock, x0 + sx - 1, y0 + r - 1, n0, sp);
+                        if (it >= npre) tma_load_4d(base + S * A_BYTES + sp * B_BYTES, &mapB, bar_full + 8 * s, cb * kKBlock, f0, tap, sp);
+                    }
                 }
+                if (++s == stages) { s = 0; ++use; }
+                if (++tap == p.taps) { tap = 0; ++cb; }
             }
         }
     } else if (warp == 1) {
@@ -482,12 +487,13 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
             constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
             bool ok = true;
+            int s = 0, use = 0;
+            const uint32_t smem_base = smem_u32(smem);
             for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % stages, use = it / stages;
                 ok = mbar_wait(bar_full + 8 * s, use & 1, status, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t base = smem_u32(smem + static_cast<size_t>(s) * STAGE_BYTES);
+                const uint32_t base = smem_base + s * STAGE_BYTES;
                 const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + A_BYTES);
                 const uint64_t b_hi = smem_desc_sw128(base + S * A_BYTES), b_lo = smem_desc_sw128(base + S * A_BYTES + B_BYTES);
 #pragma unroll
@@ -505,6 +511,7 @@ conv_umma_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     }
                 }
                 umma_commit(bar_empty + 8 * s);                 // frees the stage once these MMAs have read it
+                if (++s == stages) { s = 0; ++use; }
             }
             if (ok) umma_commit(bar_acc);
         }
@@ -671,7 +678,10 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
 
     if (warp == 0) {
         if (lane == 0) {
-            int ia = 0, ib = 0;                                  // running use counters of the two rings
+            // slots of the two rings and their use counts, advanced without divisions (this thread's instruction stream
+            // is what a short channel/tap loop waits for)
+            int sa = 0, ua = 0, sb = 0, ub = 0;
+            const uint32_t a_ring = smem_u32(smem), b_ring = smem_u32(smem_b);
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
                 int ft, x0, y0, n;
@@ -680,24 +690,22 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 for (int cb = 0; cb < KB && ok; ++cb) {
                     for (int sx = 0; sx < nshift && ok; ++sx) {
                         if constexpr (!GATHER) {
-                            const int sa = ia % NA, ua = ia / NA;
                             if (ua > 0 && !mbar_wait(bar_ea + 8 * sa, (ua - 1) & 1, status, 1)) { ok = false; break; }
-                            const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                            const uint32_t abase = a_ring + sa * a_stage;
                             mbar_expect_tx(bar_fa + 8 * sa, S * a_plane);
 #pragma unroll
                             for (int sp = 0; sp < S; ++sp)
                                 tma_load_5d(abase + sp * a_plane, &mapA, bar_fa + 8 * sa, cb * kKBlock, x0 + sx - (nshift >> 1), y0 - (nshift >> 1), n, sp);
-                            ++ia;
+                            if (++sa == NA) { sa = 0; ++ua; }
                         }
                         for (int r = 0; r < nshift; ++r) {
-                            const int sb = ib % NB, ub = ib / NB;
                             if (ub > 0 && !mbar_wait(bar_eb + 8 * sb, (ub - 1) & 1, status, 1)) { ok = false; break; }
-                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            const uint32_t bbase = b_ring + sb * b_stage;
                             mbar_expect_tx(bar_fb + 8 * sb, S * B_BYTES);
 #pragma unroll
                             for (int sp = 0; sp < S; ++sp)
                                 tma_load_4d(bbase + sp * B_BYTES, &mapB, bar_fb + 8 * sb, cb * kKBlock, f0, r * nshift + sx, sp);
-                            ++ib;
+                            if (++sb == NB) { sb = 0; ++ub; }
                         }
                     }
                 }
@@ -708,7 +716,8 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc(TERMS == 3 ? 1 : 0, BN);
             constexpr uint32_t idesc2 = instr_desc(1, MERGE ? 2 * BN : BN);
-            int ia = 0, ib = 0, j = 0;
+            int sa = 0, ua = 0, sb = 0, ub = 0, j = 0;
+            const uint32_t a_ring = smem_u32(smem), b_ring = smem_u32(smem_b);
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
                 const int buf = j & 1, ub2 = j >> 1;
@@ -717,16 +726,14 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                 bool first = true;
                 for (int cb = 0; cb < KB && ok; ++cb) {
                     for (int sx = 0; sx < nshift && ok; ++sx) {
-                        const int sa = ia % NA, ua = ia / NA;
                         ok = mbar_wait(bar_fa + 8 * sa, ua & 1, status, 2);
                         if (!ok) break;
-                        const uint32_t abase = smem_u32(smem + static_cast<size_t>(sa) * a_stage);
+                        const uint32_t abase = a_ring + sa * a_stage;
                         for (int r = 0; r < nshift && ok; ++r) {
-                            const int sb = ib % NB, ub = ib / NB;
                             ok = mbar_wait(bar_fb + 8 * sb, ub & 1, status, 2);
                             if (!ok) break;
                             tc_fence_after();
-                            const uint32_t bbase = smem_u32(smem_b + static_cast<size_t>(sb) * b_stage);
+                            const uint32_t bbase = b_ring + sb * b_stage;
                             const uint64_t b_hi = smem_desc_sw128(bbase), b_lo = smem_desc_sw128(bbase + B_BYTES);
 #pragma unroll
                             for (int mt = 0; mt < MT; ++mt) {
@@ -751,10 +758,10 @@ conv_umma_halo_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
                             }
                             first = false;
                             umma_commit(bar_eb + 8 * sb);
-                            ++ib;
+                            if (++sb == NB) { sb = 0; ++ub; }
                         }
                         if (ok) umma_commit(bar_ea + 8 * sa);
-                        ++ia;
+                        if (++sa == NA) { sa = 0; ++ua; }
                     }
                 }
                 if (ok) umma_commit(bar_af + 8 * buf);
@@ -1343,7 +1350,8 @@ void plan_dense(int F, int C, int N, int H, int W, int dtype, DensePlan &pl, boo
             if (fits && u > butil + 1e-9) { butil = u; btw = tw; }
         }
         // gathered layers: the MMA work is tiny and the kernel-side gather saves a whole tensor, so padding matters less
-        if (btw && butil >= util_now - (pl.im2col ? 0.30 : 0.02)) {
+        const double slack = debug_option("halo_slack", 2) / 100.0;   // MMA rows a halo box may waste beyond the free-form box
+        if (btw && butil >= util_now - (pl.im2col ? 0.30 : slack)) {
             const int th = kTileM / btw;
             int mt = (pl.BN == 64 && ((H + th - 1) / th) % 2 == 0) ? 2 : 1;
             if (mt == 2) {
