@@ -30,7 +30,8 @@ bool pdl_enabled();
 //   bn=N       cap of the tensor-core filter tile                  bn_keep=1 no narrowing of the filter tile
 //   ksplit=N   cluster split of the channel loop (1, 2, 4, 8)      halo=0    no persistent halo-sharing kernel
 //   mt=N       accumulator tiles per persistent CTA                pair=1    CTA-pair (cta_group::2) kernel
-//   tail=0     no K-split tail launch
+//   tail=0     no K-split tail launch                              halo_slack=N  MMA rows (%) a halo box may waste more than a free box
+//   chain=1    persistent multi-layer kernel in stacks (opt-in)    chain_stages=N  its ring depth
 // debug_option returns the integer after "key=", or dflt when the key (or the variable) is absent.
 int debug_option(const char *key, int dflt);
 bool debug_option_text(const char *key, char *buf, size_t cap);   // raw text after "key=" (false when absent)
