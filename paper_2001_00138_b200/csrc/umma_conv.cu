@@ -12,15 +12,19 @@
 // and the split rounding are below 2^-16 relative.  fp16 layers (2e-3) use one fp16 MMA on the stored values.
 //
 // Data flow.
-//   prep_act_kernel  : NCHW activations -> [S][N][H][W][Cp] (channels innermost, padded to a multiple of 64 with
-//                      zeros; S = 2 planes hi/lo for fp32 layers, 1 for fp16 layers);
-//   encode (host)    : weights -> [S][9][Fp][Cp] in the same split, zeros where pruned;
-//   conv_umma_kernel : one CTA = 128 output pixels (a TW x TH x TN box of the image batch) x BN filters.
-//       warp 0   TMA producer: per (channel block of 64, tap) loads the shifted pixel box (zero fill outside the image
-//                gives the padding) and the weight tile, 128-byte swizzle, multi-stage mbarrier ring;
-//       warp 1   one thread issues tcgen05.mma (M=128, N=BN, K=16) x 4 k-steps x 3 split terms per stage, accumulating
-//                in TMEM, and releases the stage with tcgen05.commit;
-//       warps 2-5 epilogue: tcgen05.ld the accumulator, bias + ReLU, store NCHW.
+//   transition_* kernels  : NCHW activations -> [S][N][H][W][Cp] (channels innermost, padded to a multiple of 64 with
+//                           zeros; S = 2 planes hi/lo for fp32 layers, 1 for fp16 layers); inside a stack the previous
+//                           layer's epilogue writes this tensor instead;
+//   encode (host)         : weights -> [S][9][Fp][Cp] in the same split, zeros where pruned;
+//   conv_umma_kernel      : one CTA = 128 output pixels (a TW x TH x TN box of the image batch) x BN filters; small grids
+//                           split the channel/tap loop over a thread-block cluster;
+//   conv_umma_halo_kernel : persistent CTAs, three halo boxes per channel block instead of nine, double-buffered TMEM.
+//       warp 0     TMA producer: per (channel block of 64, tap) the shifted pixel box (zero fill outside the image gives
+//                  the padding) and the weight tile, 128-byte swizzle, mbarrier rings;
+//       warp 1     one thread issues tcgen05.mma (M=128, K=16, 4 k-steps per stage, the split products) into TMEM and
+//                  releases the stage with tcgen05.commit;
+//       warps 2-9  epilogue: tcgen05.ld the accumulator, bias + ReLU (+ 2x2 maximum), store NCHW or the next layer's
+//                  operands.
 // Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves through the normal exit
 // (TMEM is always deallocated).  Every TMA load is issued by, and lands in, one CTA only.
 #include <cuda.h>

@@ -496,3 +496,31 @@ def test_random_stacks(seed):
     stack.free()
     for hd in handles:
         hd.free()
+
+
+@pytest.mark.parametrize("C,prune", [(1, 0.0), (3, 0.75), (5, 0.8), (7, 0.9)])
+def test_auto_keeps_few_channel_fp32_layers_exact_whatever_the_pattern_set(C, prune):
+    """Few input channels, heavy pruning and a pattern set outside the tiled kernel's built-in table: with one or two
+    products per output the hi/lo split of the tensor-core path would sit at the edge of 1e-4, so AUTO must keep such
+    fp32 layers on an FP32 kernel (here the generic FKW kernel), and the result must hold the tolerance."""
+    rng = np.random.Generator(np.random.PCG64(4000 + C))
+    pats = np.asarray([0b000101011, 0b110100010, 0b011000101, 0b101010001], dtype=np.uint16)   # four 4-of-9 masks, none built in
+    assert all(bin(int(m)).count("1") == 4 for m in pats) and not set(int(m) for m in pats) & set(synth.PATTERN_MASKS)
+    N, F, H, W = 2, 48, 19, 23
+    w = rng.standard_normal((F, C, 3, 3)).astype(np.float32) * 3.0
+    pid = rng.integers(0, len(pats), size=(F, C)).astype(np.int32)
+    pid[rng.random((F, C)) < prune] = -1
+    mask = synth.mask_from_pid(pid, pats)
+    bias = (rng.standard_normal(F) * 0.2).astype(np.float32)
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    layer = B.encode(w, mask, pats, N=N, H=H, W=W, relu=False, bias=bias)
+    assert layer.plan()["variant"] in (VARIANTS["reorder"], VARIANTS["tiled"]), "not the tensor-core variant"
+    out = torch.full((N, F, H, W), float("nan"), device="cuda")
+    layer.conv(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
+    layer.check()
+    layer.free()
+    assert_close(out.cpu().numpy(), oracle.conv3x3(x, w, mask, bias, False), TOL_F32, f"AUTO, C={C}, prune={prune}")
+
