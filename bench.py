@@ -258,7 +258,7 @@ def run_suite(args):
     ALU_PEAK_TFLOPS = alu_peak_tflops(torch)
     stream = torch.cuda.current_stream().cuda_stream
     flush = torch.empty(256 * 1024 * 1024 // 4, device="cuda")
-    variants = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense_tc": 4}
+    variants = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense_tc": 4, "pattern_run": 5}
 
     def measure(tag, L, N, variant="auto", order=None, reps=20):
         dt = B.F16 if L.dtype == "f16" else B.F32
@@ -278,10 +278,11 @@ def run_suite(args):
         plan = h.plan()
         print(json.dumps({"suite": tag, "layer": L.name, "batch": N, "variant": variant,
                           "kernel": "generated_fp32" if plan.get("generated") else
-                                    {1: "noopt", 2: "reorder", 3: "tiled", 4: "dense_tc"}[plan["variant"]],
+                                    {1: "noopt", 2: "reorder", 3: "tiled", 4: "dense_tc", 5: "pattern_run"}[plan["variant"]],
                           "filter_order": "random" if order is not None else "fkr", "K": L.K,
                           "us": round(us, 2), "gflops_nonzero": round(flops / us / 1e3, 1),
                           "roofline_us": round(roof_us, 2), "bound": bound, "frac": round(roof_us / us, 3),
+                          "lane_use": round(L.K / plan["entries"], 3) if plan["variant"] == 5 else None,
                           "l2": "flushed between launches" if small else "working set larger than L2"}), flush=True)
         h.free()
 
@@ -300,6 +301,17 @@ def run_suite(args):
                 measure("sweep", L, 64, order=synth.random_filter_order(512, 7))
                 measure("sweep", L, 64, variant="tiled")
                 measure("sweep", L, 64, variant="tiled", order=synth.random_filter_order(512, 7))
+                measure("sweep", L, 64, variant="pattern_run")
+                measure("sweep", L, 64, variant="pattern_run", order=synth.random_filter_order(512, 7))
+    if "crossover" in which or "all" in which:
+        # beyond the baseline's sweep: where the kernel whose time follows the kept kernels overtakes the dense tensor-core path
+        for npat in (4, 8, 12):
+            for prune in (0.95, 0.97, 0.99):
+                L = synth.make_layer(f"sweep_p{npat}_prune{int(prune * 100)}", F=512, C=512, N=64, H=14, W=14, seed=5100 + npat,
+                                     n_patterns=npat, prune=prune, draw_input=False)
+                for variant in ("auto", "dense_tc", "pattern_run"):
+                    measure("crossover", L, 64, variant=variant)
+                measure("crossover", L, 64, variant="pattern_run", order=synth.random_filter_order(512, 7))
     if "cifar" in which or "all" in which:
         suite_cifar_stack(B, synth, torch, hbm, stream)
     if "storage" in which or "all" in which:
@@ -458,7 +470,7 @@ def main():
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
     ap.add_argument("--suite", default="", help="instead of the headline step: cfg2,resnet,sweep,ablation,cifar,storage,context or all "
-                                                "(one JSON line per measured point)")
+                                                "(one JSON line per measured point); also: crossover")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -71,16 +71,21 @@ enum { PATDNN_F32 = 0, PATDNN_F16 = 1 };   /* storage type of weights and activa
  * the first layer of the VGG-16 and ResNet-50 shaped workloads -- and, for layers with at most 4 input channels and 64
  * filters, FP32 code generated for the layer at run time (kept weights as immediates; the tiled kernel where no
  * run-time compiler is present).  Other few-channel fp32 layers stay on TILED, or on REORDER when their pattern set
- * is not among the tiled kernel's twelve built-in patterns.  The explicit values run the kernel they name and exist
- * for the ablation ladder of Section 6.3 (no optimisation -> +reorder -> +load-redundancy elimination -> tensor
+ * is not among the tiled kernel's twelve built-in patterns.  Layers that keep at most ~1 kernel in 7 are also planned
+ * for PATTERN_RUN, whose time follows the kept kernels, and take it where its estimate clearly beats the others (on the
+ * 512 -> 512 @ 14x14 sweep layer: from ~96 % connectivity pruning on).  The explicit values run the kernel they name and
+ * exist for the ablation ladder of Section 6.3 (no optimisation -> +reorder -> +load-redundancy elimination -> tensor
  * cores). */
 enum {
     PATDNN_VARIANT_AUTO = 0,
     PATDNN_VARIANT_NOOPT = 1,     /* original filter order, per-kernel branch on the pattern, global loads */
     PATDNN_VARIANT_REORDER = 2,   /* walks the FKW arrays in pattern order (branch-free per run), global loads */
     PATDNN_VARIANT_TILED = 3,     /* shared-memory tile + halo, register patch reuse across taps and filters */
-    PATDNN_VARIANT_DENSE_TC = 4   /* per-tap dense implicit GEMM on the tensor cores (tcgen05); fp32 layers use three
+    PATDNN_VARIANT_DENSE_TC = 4,  /* per-tap dense implicit GEMM on the tensor cores (tcgen05); fp32 layers use three
                                      bf16 products of operands split into hi + lo; chosen where it beats TILED */
+    PATDNN_VARIANT_PATTERN_RUN = 5 /* one filter per lane, the FKW pattern runs of Section 5.3 as warp-uniform step lists,
+                                     the whole input tile (all channels) in shared memory; its time follows the number
+                                     of kept kernels; AUTO takes it for very sparse layers on small images */
 };
 
 enum { PATDNN_FLAG_HOST_ONLY = 1 };   /* encode on the host only: no device is touched, patdnn_conv is refused */
@@ -119,6 +124,10 @@ PATDNN_API int patdnn_encode(const float *weights, const uint8_t *mask, const ui
  * `stream`, with the kernel the handle was planned for:
  *   TILED     shared-memory tile + halo staging, pattern-ordered branch-free FMA bodies, register patch reused by the
  *             four taps of a kernel and by the filters of a warp (Sections 5.2 and 5.4), output scattered through reorder[];
+ *   PATTERN_RUN  one filter per lane: the filter's FKW pattern runs (stride[], Section 5.3) as warp-uniform step lists, the
+ *             channel of a kernel an indirect shared-memory address, one unrolled body per pattern that streams the
+ *             patch rows through registers; the whole input tile (all channels) in shared memory: needs built-in
+ *             patterns and (C + 1) * 324 bytes <= 200 KB;
  *   REORDER / NOOPT  the generic kernels of the ablation ladder (any pattern set);
  *   DENSE_TC  one layout kernel (NCHW -> channels-innermost, operands split into bf16 hi + lo for fp32 layers) into a
  *             handle-owned scratch buffer, then the tcgen05 implicit GEMM over nine shifted TMA boxes (one launch, plus a

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(HERE, "libpatdnn.so")
 
 OK = 0
 F32, F16 = 0, 1
-VARIANT_AUTO, VARIANT_NOOPT, VARIANT_REORDER, VARIANT_TILED, VARIANT_DENSE_TC = 0, 1, 2, 3, 4
+VARIANT_AUTO, VARIANT_NOOPT, VARIANT_REORDER, VARIANT_TILED, VARIANT_DENSE_TC, VARIANT_PATTERN_RUN = 0, 1, 2, 3, 4, 5
 FLAG_HOST_ONLY = 1
 STATUS_NAMES = {0: "OK", 1: "E_NULL", 2: "E_SHAPE", 3: "E_PATTERN_SET", 4: "E_MASK", 5: "E_ORDER", 6: "E_CUDA",
                 7: "E_NO_DEVICE", 8: "E_DEVICE_TIMEOUT", 9: "E_DTYPE", 10: "E_ALLOC", 11: "E_STACK", 12: "E_SCRATCH"}

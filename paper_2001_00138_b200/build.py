@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatdnn.so")
-SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "umma_chain.cu", "smallc_split.cu", "smallc_jit.cu", "tiled_inst_4x8.cu",
+SOURCES = ["api.cu", "kernels_simple.cu", "kernels_tiled.cu", "umma_conv.cu", "umma_chain.cu", "prun_conv.cu", "prun_plan.cpp", "smallc_split.cu", "smallc_jit.cu", "tiled_inst_4x8.cu",
            "tiled_inst_4x4.cu", "tiled_inst_2x8.cu", "fkw_encoder.cpp", "tiled_plan.cpp"]
 HEADERS = ["kernels.hpp", "umma_ptx.cuh", "kernels_tiled.cuh", "fkw_encoder.hpp", os.path.join("generated", "tiled_cases.inc"),
            os.path.join("..", "..", "include", "patdnn.h")]

@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -66,6 +67,11 @@ struct patdnn_layer {
     uint32_t *d_rec = nullptr;
     int32_t *d_seg = nullptr, *d_seglen = nullptr;
     int64_t device_bytes = 0;
+    // pattern-run kernel
+    PrunPlan prun;
+    uint32_t *d_prun_chan = nullptr;
+    float *d_prun_wts = nullptr;
+    int32_t *d_prun_runs = nullptr;
     // dense tensor-core path
     DensePlan dense;
     uint16_t *d_wdense = nullptr;
@@ -161,7 +167,7 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
     if (desc->F < 1 || desc->C < 1 || desc->N < 0 || desc->H < 1 || desc->W < 1) return PATDNN_E_SHAPE;
     if (desc->H > 65535 || desc->W > 65535 || desc->N > 65535) return PATDNN_E_SHAPE;
     if (desc->dtype != PATDNN_F32 && desc->dtype != PATDNN_F16) return PATDNN_E_DTYPE;
-    if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_DENSE_TC) return PATDNN_E_DTYPE;
+    if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_PATTERN_RUN) return PATDNN_E_DTYPE;
     if (desc->filter_order != 0 && desc->filter_order != 1) return PATDNN_E_ORDER;
     if (desc->filter_order == 1 && !desc->order) return PATDNN_E_NULL;
     patdnn_layer *h = new (std::nothrow) patdnn_layer();
@@ -182,33 +188,54 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                 h->variant = can_tile ? PATDNN_VARIANT_TILED : PATDNN_VARIANT_REORDER;
                 // Tensor cores only where the dense reformulation is expected to win: compare a time estimate of the
                 // zero-padded per-tap GEMMs with the CUDA-core kernel's rate on the kept weights (both measured on
-                // B200: ~900 TFLOP/s sustained for the 16-bit MMAs of this kernel, ~12 TFLOP/s for the tiled kernel).
+                // B200: ~1200 TFLOP/s sustained for the 16-bit MMAs of this kernel, ~12 TFLOP/s for the tiled kernel).
                 if (!(desc->flags & PATDNN_FLAG_HOST_ONLY) && desc->N > 0 &&
                     dense_supported(desc->F, desc->C, desc->N, desc->H, desc->W)) {
                     DensePlan dp;
                     plan_dense(desc->F, desc->C, desc->N, desc->H, desc->W, desc->dtype, dp);
                     const double terms = desc->dtype == PATDNN_F16 ? 1.0 : 3.0;
                     const double rows = static_cast<double>(dp.tiles_x) * dp.tiles_y * dp.tiles_n * 128.0;
-                    const double t_dense = terms * 2.0 * dp.taps * dp.Cp * dp.Fp * rows / 9.0e14 +
+                    const double t_dense = terms * 2.0 * dp.taps * dp.Cp * dp.Fp * rows / 1.2e15 +
                                            static_cast<double>(desc->N) * desc->H * desc->W * (desc->C * 4.0 + dp.Cp * 2.0 * dp.S) / 4.0e12 +
                                            4e-6;
                     // CUDA-core kernel: ~12 TFLOP/s on kept weights for large images, ~4 for 14x14-class layers (measured)
                     const double tiled_rate = (desc->H * desc->W <= 256) ? 4.0e12 : 1.2e13;
-                    const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / tiled_rate + 1.5e-5;
+                    // (every CTA of the tiled kernel's filter dimension -- 16 filters each -- stages the whole input again)
+                    const double t_tiled = 8.0 * h->fkw.K * static_cast<double>(desc->N) * desc->H * desc->W / tiled_rate + 1.5e-5 +
+                                           std::ceil(desc->F / 16.0) * desc->N * desc->C * static_cast<double>(desc->H) * desc->W *
+                                               (desc->dtype == PATDNN_F16 ? 2.0 : 4.0) / 3.5e12;
                     // layers with 9*C <= 64 (gathered-neighbourhood GEMM) are store-bound there: measured slower than the
                     // CUDA-core kernel on the RGB first layer, so AUTO leaves them on it unless it cannot run the layer
                     // (when the tiled kernel cannot take such a layer -- a pattern outside its builtin table -- fp32 layers
                     // go to the generic FKW kernel, which is exact to fp32: with so few terms per output the hi/lo split's
                     // per-product error is not averaged down)
                     if (t_dense < t_tiled && (!dp.im2col || (!can_tile && desc->dtype == PATDNN_F16))) h->variant = PATDNN_VARIANT_DENSE_TC;
+                    // Very sparse layers: the pattern-run kernel's time follows the kept kernels (measured with 16 warps per
+                    // CTA: ~0.8 us per step of the slowest warp plus ~20 us per wave of CTAs), the tensor cores' does
+                    // not.  Worth planning only where it can win: at most ~1 in 7 kernels kept.
+                    if (static_cast<double>(h->fkw.K) <= 0.15 * desc->F * desc->C && prun_supported(h->fkw, desc->N, desc->H, desc->W)) {
+                        PrunPlan pp;
+                        PrunLayout pl_tmp;
+                        if (plan_prun(h->fkw, desc->N, desc->H, desc->W, pp, pl_tmp) == PATDNN_OK) {
+                            const double ctas = static_cast<double>(desc->N) * pp.tiles_x * pp.tiles_y * pp.groups;
+                            const double waves = std::ceil(ctas / sm_count());
+                            const double t_prun = waves * (pp.max_warp_steps * (0.055e-6 * pp.groups_per_cta) + 25e-6);
+                            const double t_best = h->variant == PATDNN_VARIANT_DENSE_TC ? t_dense : t_tiled;
+                            if (t_prun < 0.8 * t_best) h->variant = PATDNN_VARIANT_PATTERN_RUN;   // clear wins only
+                        }
+                    }
                 }
             } else {
                 h->variant = desc->variant;
             }
             if (desc->N == 0) h->variant = PATDNN_VARIANT_REORDER;   // an empty batch launches nothing: no plan to make
             if (h->variant == PATDNN_VARIANT_TILED && !can_tile) rc = PATDNN_E_SHAPE;
+            if (h->variant == PATDNN_VARIANT_PATTERN_RUN && !prun_supported(h->fkw, desc->N, desc->H, desc->W)) rc = PATDNN_E_SHAPE;
         }
         TiledLayout lay;
+        PrunLayout play;
+        if (rc == PATDNN_OK && h->variant == PATDNN_VARIANT_PATTERN_RUN)
+            rc = plan_prun(h->fkw, desc->N, desc->H, desc->W, h->prun, play);
         if (rc == PATDNN_OK && h->variant == PATDNN_VARIANT_TILED)
             rc = plan_tiled(h->fkw, desc->N, desc->H, desc->W, desc->dtype, h->plan, lay);
         if (rc == PATDNN_OK && !(desc->flags & PATDNN_FLAG_HOST_ONLY)) {
@@ -252,6 +279,17 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                     if (!rc) {
                         cudaError_t pe = prepare_dense(h->dense, desc->dtype);
                         if (pe != cudaSuccess) rc = cuda_fail(pe, "cudaFuncSetAttribute(dense kernel)");
+                    }
+                } else if (h->variant == PATDNN_VARIANT_PATTERN_RUN) {
+                    rc = upload(play.chan, &h->d_prun_chan, h->owned);
+                    if (!rc) rc = upload(play.wts, &h->d_prun_wts, h->owned);
+                    if (!rc) rc = upload(play.run_ofs, &h->d_prun_runs, h->owned);
+                    if (!rc) rc = upload(k.reorder, &h->d_reorder, h->owned);
+                    if (!rc) rc = upload(h->bias, &h->d_bias, h->owned);
+                    h->device_bytes = static_cast<int64_t>(play.chan.size()) * 4 + play.wts.size() * 4 + play.run_ofs.size() * 4 + k.F * 8;
+                    if (!rc) {
+                        cudaError_t pe = prepare_prun(h->prun, desc->dtype);
+                        if (pe != cudaSuccess) rc = cuda_fail(pe, "cudaFuncSetAttribute(shared memory)");
                     }
                 } else if (h->variant == PATDNN_VARIANT_TILED) {
                     rc = upload(lay.rec, &h->d_rec, h->owned);
@@ -315,6 +353,14 @@ int patdnn_conv(patdnn_handle h, const void *in, void *out, void *stream) {
         e = smallc_jit_launch(h->jit_nchw, in, out, d.N, d.H, d.W, st);
     } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         return dense_forward(h, h->dense, in, h->d_act, out, st);
+    } else if (h->variant == PATDNN_VARIANT_PATTERN_RUN) {
+        PrunParams p{};
+        p.in = in; p.out = out;
+        p.chan = h->d_prun_chan; p.wts = h->d_prun_wts; p.run_ofs = h->d_prun_runs; p.reorder = h->d_reorder; p.bias = h->d_bias;
+        p.N = d.N; p.C = d.C; p.H = d.H; p.W = d.W; p.F = d.F; p.P = h->fkw.P;
+        p.tiles_x = h->prun.tiles_x; p.tiles_y = h->prun.tiles_y; p.relu = d.relu; p.groups_per_cta = h->prun.groups_per_cta;
+        std::memcpy(p.builtin, h->prun.builtin, sizeof p.builtin);
+        e = launch_prun(h->prun, p, d.dtype, st);
     } else if (h->variant == PATDNN_VARIANT_TILED) {
         TiledParams p{};
         p.in = in; p.out = out;
@@ -466,6 +512,13 @@ int patdnn_plan(patdnn_handle h, patdnn_plan_info *info) {
         info->grid_x = p.grid_pix * p.grid_fg; info->grid_y = 1; info->grid_z = 1;
         info->smem_bytes = p.smem_bytes;
         info->entries = p.entries;
+    } else if (h->variant == PATDNN_VARIANT_PATTERN_RUN) {
+        const PrunPlan &p = h->prun;
+        info->tile_rows = kPrunTile; info->tile_cols = kPrunTile; info->filters_per_warp = 32;
+        info->warps_per_cta = p.threads / 32; info->channels_per_stage = h->desc.C; info->channel_splits = 1;
+        info->grid_x = h->desc.N * p.tiles_y * p.tiles_x; info->grid_y = p.groups; info->grid_z = 1;
+        info->smem_bytes = p.smem_bytes;
+        info->entries = p.entries;                               // lane entries, padding included: kept kernels / entries = lane use
     } else if (h->variant == PATDNN_VARIANT_DENSE_TC) {
         const DensePlan &p = h->dense;
         info->tile_rows = p.TH * p.MT; info->tile_cols = p.TW; info->filters_per_warp = p.BN; info->warps_per_cta = 10;

@@ -138,6 +138,41 @@ int plan_tiled(const Fkw &fkw, int N, int H, int W, int dtype, TiledPlan &plan, 
 cudaError_t launch_tiled(const TiledPlan &plan, const TiledParams &p, int dtype, cudaStream_t stream);
 cudaError_t prepare_tiled(const TiledPlan &plan, int dtype);   // opt in to the dynamic shared memory size
 
+// ---- pattern-run kernel: one filter per lane, FKW pattern runs as step lists (prun_conv.cu, prun_plan.cpp) ---------------
+constexpr int kPrunTile = 7;          // output pixels per thread: 7 x 7
+constexpr int kPrunWarps = 16;        // warps per CTA, one per warp group of 32 filters
+struct PrunPlan {
+    int tiles_x = 0, tiles_y = 0;     // 7 x 7 tiles per image
+    int groups = 0, threads = 0;      // filter groups of up to 512 positions (grid.y); threads per CTA
+    int groups_per_cta = 0;           // warp groups a CTA holds (at most 16)
+    int smem_bytes = 0;
+    int builtin[32] = {};             // per pattern of the layer: its index in the built-in pattern table
+    int64_t steps = 0, entries = 0;   // warp steps over all groups; lane entries (32 per step, padding included)
+    int max_warp_steps = 0;           // steps of the slowest warp (two groups each): what a CTA waits for
+};
+struct PrunLayout {                   // host image of the private device layout
+    std::vector<int32_t> run_ofs;     // [warp groups][P + 1] first step of each pattern run
+    std::vector<uint32_t> chan;       // [steps][32] word offset of the lane's channel patch in shared memory
+    std::vector<float> wts;           // [steps][4][32] the kernel's four kept weights (ascending tap order)
+};
+struct PrunParams {
+    const void *in;
+    void *out;
+    const uint32_t *chan;
+    const float *wts;
+    const int32_t *run_ofs;
+    const int32_t *reorder;
+    const float *bias;
+    int N, C, H, W, F, P;
+    int tiles_x, tiles_y, relu;
+    int groups_per_cta;               // warp groups (of the 16 a CTA can hold) that exist: ceil(min(F, 512) / 32)
+    int builtin[32];
+};
+bool prun_supported(const Fkw &fkw, int N, int H, int W);
+int plan_prun(const Fkw &fkw, int N, int H, int W, PrunPlan &plan, PrunLayout &layout);
+cudaError_t prepare_prun(const PrunPlan &plan, int dtype);
+cudaError_t launch_prun(const PrunPlan &plan, const PrunParams &p, int dtype, cudaStream_t stream);
+
 // ---- dense tensor-core reformulation (umma_conv.cu) -----------------------------------------------------------
 struct DensePlan {
     int S = 0;                  // operand planes: 2 (bf16 hi + lo, fp32 layers) or 1 (fp16 layers)

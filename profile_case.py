@@ -64,7 +64,7 @@ def main():
     ap.add_argument("--layer", default="vgg6")
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--reps", type=int, default=3)
-    ap.add_argument("--variant", default="auto", choices=["auto", "noopt", "reorder", "tiled", "dense"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "noopt", "reorder", "tiled", "dense", "prun"])
     ap.add_argument("--chain", type=int, default=1)
     args = ap.parse_args()
     import torch
@@ -77,7 +77,7 @@ def main():
     N = L.N if args.layer in ("cfg1", "cfg2") else args.batch
     dt = B.F16 if L.dtype == "f16" else B.F32
     tdt = torch.float16 if L.dtype == "f16" else torch.float32
-    variant = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense": 4}[args.variant]
+    variant = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense": 4, "prun": 5}[args.variant]
     h = B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, dtype=dt, relu=True, bias=L.bias, variant=variant)
     x = torch.rand((N, L.C, L.H, L.W), device="cuda").to(tdt)
     y = torch.empty((N, L.F, L.H, L.W), device="cuda", dtype=tdt)

@@ -18,10 +18,10 @@ def _lib():
     return binding
 
 
-VARIANTS = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense": 4}
+VARIANTS = {"auto": 0, "noopt": 1, "reorder": 2, "tiled": 3, "dense": 4, "prun": 5}
 
 
-@pytest.mark.parametrize("variant", ["tiled", "dense", "reorder", "noopt"])
+@pytest.mark.parametrize("variant", ["tiled", "dense", "reorder", "noopt", "prun"])
 def test_config1(variant):
     L = synth.config1()
     got, plan = gpu_layer(L, variant=VARIANTS[variant])
@@ -40,9 +40,11 @@ ODD_SHAPES = [
 
 
 @pytest.mark.parametrize("shape", ODD_SHAPES)
-@pytest.mark.parametrize("variant", ["tiled", "dense", "reorder"])
+@pytest.mark.parametrize("variant", ["tiled", "dense", "reorder", "prun"])
 def test_odd_shapes(shape, variant):
     N, C, F, H, W, npat, prune = shape
+    if variant == "prun" and C > 600:
+        pytest.skip("the pattern-run kernel keeps all channels of a 9 x 9 patch in shared memory: C <= ~630")
     L = synth.make_layer("odd", F=F, C=C, N=N, H=H, W=W, seed=hash(shape) % 10000, n_patterns=npat, prune=prune,
                          bias_std=0.2, x_dist="normal", relu=(F % 2 == 1))
     got, _ = gpu_layer(L, variant=VARIANTS[variant])
@@ -60,7 +62,7 @@ def test_empty_filters_and_caller_order():
     L.mask[3] = 0
     L.mask[17] = 0
     ref = oracle_layer(L)
-    for variant in ("tiled", "dense", "reorder"):
+    for variant in ("tiled", "dense", "reorder", "prun"):
         got, _ = gpu_layer(L, variant=VARIANTS[variant])
         assert_close(got, ref, TOL_F32, variant)
         assert np.all(got[:, 3] == max(L.bias[3], 0.0))
@@ -105,7 +107,7 @@ def test_resnet_shapes_fp16(i, N):
     """The four ResNet-50-shaped fp16 layers at batch 1, a ragged batch and the full batch of 32, whole output."""
     L = synth.resnet50_layer(i, N=N)
     ref = oracle_layer(L)
-    for variant in ("auto", "tiled", "dense", "reorder"):
+    for variant in ("auto", "tiled", "dense", "reorder", "prun"):
         if N == 32 and variant == "reorder":
             continue                      # the generic kernel adds nothing at full batch
         if variant == "tiled" and L.W % 2:
@@ -172,7 +174,7 @@ def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype, g
 def test_sweep_points_reduced_batch(npat, prune):
     L = synth.sweep_layer(npat, prune, N=3)
     ref = oracle_layer(L)
-    for variant in ("auto", "tiled", "dense"):
+    for variant in ("auto", "tiled", "dense", "prun"):
         got, _ = gpu_layer(L, variant=VARIANTS[variant])
         assert_close(got, ref, TOL_F32, f"sweep p{npat} prune{prune} {variant}")
     got, _ = gpu_layer(L, order=synth.random_filter_order(512, 1))
@@ -185,9 +187,10 @@ def test_sweep_points_full_batch(npat, prune):
     filter reorder and with a seeded random filter order."""
     L = synth.sweep_layer(npat, prune, N=64)
     ref = oracle_layer(L)
-    for variant in ("auto", "tiled"):
-        got, _ = gpu_layer(L, variant=VARIANTS[variant])
+    for variant in ("auto", "tiled", "prun"):
+        got, plan = gpu_layer(L, variant=VARIANTS[variant])
         assert_close(got, ref, TOL_F32, f"sweep N=64 p{npat} prune{prune} {variant}")
+    assert plan["variant"] == VARIANTS["prun"] and plan["entries"] >= L.K, "lane entries = kept kernels + padding"
     got, _ = gpu_layer(L, order=synth.random_filter_order(512, 7))
     assert_close(got, ref, TOL_F32, f"sweep N=64 p{npat} prune{prune} random filter order")
 
@@ -395,7 +398,7 @@ def test_empty_batch_is_a_no_op():
     import torch
     from paper_2001_00138_b200 import binding as B
     L = synth.make_layer("z", F=16, C=8, N=1, H=6, W=6, seed=3, draw_input=False)
-    for variant in ("auto", "dense", "tiled", "reorder"):
+    for variant in ("auto", "dense", "tiled", "reorder", "prun"):
         h = B.encode(L.weights, L.mask, L.patterns, N=0, H=6, W=6, relu=True, bias=L.bias, variant=VARIANTS[variant])
         x = torch.empty((0, 8, 6, 6), device="cuda")
         y = torch.empty((0, 16, 6, 6), device="cuda")
@@ -453,7 +456,7 @@ def test_random_layers_all_planner_paths(case):
                          x_dist="normal", dtype=dtype, relu=relu)
     ref = oracle_layer(L)
     tol = TOL_F16 if dtype == "f16" else TOL_F32
-    for variant in ("auto", "dense"):
+    for variant in ("auto", "dense", "prun"):
         got, _ = gpu_layer(L, variant=VARIANTS[variant])
         assert_close(got, ref, tol, f"{case}/{variant}")
 
