@@ -158,3 +158,23 @@ def test_patterns_outside_the_builtin_table_fall_back_to_the_generic_kernel(B):
     with pytest.raises(B.PatdnnError):
         B.encode(w, mask, pats, N=1, H=8, W=8, variant=B.VARIANT_TILED, host_only=True)
     layer.free()
+
+
+def test_pattern_run_step_lists_cover_every_kept_kernel():
+    """Host side of the pattern-run kernel: the warp-uniform step lists hold every kept kernel once plus zero-weight
+    padding (whole steps of 32 lanes); a layer whose input tile cannot stay in shared memory is refused."""
+    from paper_2001_00138_b200 import binding as B, synth
+    for F, C, prune in ((70, 40, 0.8), (512, 96, 0.9), (33, 7, 0.0)):
+        L = synth.make_layer("steps", F=F, C=C, N=2, H=9, W=11, seed=F + C, prune=prune, draw_input=False)
+        h = B.encode(L.weights, L.mask, L.patterns, N=2, H=9, W=11, variant=B.VARIANT_PATTERN_RUN, host_only=True)
+        p = h.plan()
+        h.free()
+        assert p["variant"] == B.VARIANT_PATTERN_RUN and p["tile_rows"] == 7 and p["tile_cols"] == 7
+        assert p["entries"] % 32 == 0 and p["entries"] >= L.K
+        if prune == 0.0:
+            assert p["entries"] <= 1024                            # 231 kernels: two warp groups, the second with one filter
+    L = synth.make_layer("wide", F=16, C=700, N=1, H=7, W=7, seed=3, prune=0.5, draw_input=False)
+    with pytest.raises(B.PatdnnError) as e:
+        B.encode(L.weights, L.mask, L.patterns, N=1, H=7, W=7, variant=B.VARIANT_PATTERN_RUN, host_only=True)
+    assert e.value.status == 2
+
