@@ -113,6 +113,9 @@ typedef struct {
  *   pattern_set  HOST uint16 [n_patterns] 9-bit masks, 1 <= n_patterns <= 32
  *   desc         HOST; copied
  *   out          receives the handle on success (untouched on failure)
+ * Size limits (E_SHAPE beyond them): F, N, H, W <= 65535; max(C, F) * H * W < 2^31 (one image's input and output; the
+ * whole batch may hold more than 2^31 elements); PATDNN_VARIANT_DENSE_TC additionally H, W <= 4096 and
+ * N * ceil(C / 64) <= 65535 (AUTO falls back to a CUDA-core variant beyond that).
  * Errors: E_NULL, E_SHAPE, E_PATTERN_SET, E_MASK, E_ORDER, E_DTYPE, E_ALLOC, E_CUDA.
  * The call is synchronous (it returns after the upload completed) and uses the current CUDA device.
  */

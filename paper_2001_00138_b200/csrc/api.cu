@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstdint>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -165,7 +166,10 @@ int patdnn_encode(const float *weights, const uint8_t *mask, const uint16_t *pat
                   const patdnn_desc *desc, patdnn_handle *out) {
     if (!weights || !mask || !pattern_set || !desc || !out) return PATDNN_E_NULL;
     if (desc->F < 1 || desc->C < 1 || desc->N < 0 || desc->H < 1 || desc->W < 1) return PATDNN_E_SHAPE;
-    if (desc->H > 65535 || desc->W > 65535 || desc->N > 65535) return PATDNN_E_SHAPE;
+    if (desc->H > 65535 || desc->W > 65535 || desc->N > 65535 || desc->F > 65535) return PATDNN_E_SHAPE;
+    // one image's input and output each stay below 2^31 elements (offsets inside an image are 32-bit; the batch is not
+    // limited that way: offsets that include the image index are 64-bit)
+    if (static_cast<int64_t>(std::max(desc->C, desc->F)) * desc->H * desc->W > INT32_MAX) return PATDNN_E_SHAPE;
     if (desc->dtype != PATDNN_F32 && desc->dtype != PATDNN_F16) return PATDNN_E_DTYPE;
     if (desc->variant < PATDNN_VARIANT_AUTO || desc->variant > PATDNN_VARIANT_PATTERN_RUN) return PATDNN_E_DTYPE;
     if (desc->filter_order != 0 && desc->filter_order != 1) return PATDNN_E_ORDER;

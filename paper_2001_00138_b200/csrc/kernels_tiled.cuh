@@ -129,7 +129,9 @@ __global__ void __launch_bounds__(PW *FW * 32, MINB) conv_tiled_kernel(const Til
     int2 *s_items = reinterpret_cast<int2 *>(smem + NS * stage_b);
 
     // Copy plan of one channel, built once: for every copy group of every staged row, the source element offset
-    // inside a channel plane (image offset included; -1 = zero fill) and the destination byte offset.
+    // inside a channel plane (counted from the first image this CTA stages, so that it fits 32 bits whatever the
+    // batch; -1 = zero fill) and the destination byte offset.
+    const int n_base = vr_lo / (p.H + 2);
     {
         const int epg = p.copy_bytes / ES;
         for (int i = tid; i < nitems; i += NT) {
@@ -138,7 +140,7 @@ __global__ void __launch_bounds__(PW *FW * 32, MINB) conv_tiled_kernel(const Til
             const int nn = vr / (p.H + 2), yy = vr - nn * (p.H + 2) - 1;
             const int col = g * epg - p.lead;
             const bool ok = nn < p.N && yy >= 0 && yy < p.H && col >= 0 && col < p.W;
-            s_items[i] = make_int2(ok ? (nn * p.C * p.H + yy) * p.W + col : -1, row * pitch_b + g * p.copy_bytes);
+            s_items[i] = make_int2(ok ? ((nn - n_base) * p.C * p.H + yy) * p.W + col : -1, row * pitch_b + g * p.copy_bytes);
         }
     }
     if (tid < NS * 4)   // the zero group behind each stage's input rows (read as "column W" of the very last row)
@@ -153,7 +155,7 @@ __global__ void __launch_bounds__(PW *FW * 32, MINB) conv_tiled_kernel(const Til
         const uint32_t sin = smem_u32(smem + s * stage_b);
         const int c0 = q * p.CC;
         const int ccn = min(p.CC, p.C - c0);
-        const T *gchunk = gin + static_cast<size_t>(c0) * plane;
+        const T *gchunk = gin + (static_cast<size_t>(n_base) * p.C + c0) * plane;
         for (int i = tid; i < nitems; i += NT) {
             const int2 it = s_items[i];
             const bool ok = it.x >= 0;

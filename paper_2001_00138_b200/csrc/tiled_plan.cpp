@@ -46,7 +46,8 @@ bool tiled_supported(const Fkw &fkw, int N, int H, int W, int dtype) {
     for (uint16_t m : fkw.patterns)
         if (builtin_id(m) < 0) return false;
     if (row_copy_bytes(W, dtype) == 0) return false;
-    if (static_cast<int64_t>(N) * std::max(fkw.C, fkw.F) * H * W >= (int64_t(1) << 31)) return false;
+    if (static_cast<int64_t>(std::max(fkw.C, fkw.F)) * H * W >= (int64_t(1) << 31)) return false;   // 32-bit offsets inside one image
+    if (static_cast<int64_t>(N) * (H + 2) >= (int64_t(1) << 31) || static_cast<int64_t>(N) * H * W >= (int64_t(1) << 33)) return false;
     if (W > 1024) return false;
     return true;
 }

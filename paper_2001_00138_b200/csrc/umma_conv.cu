@@ -1270,7 +1270,10 @@ int cluster_capacity(int bn, int dtype, int ks, int smem) {
 }  // namespace
 
 bool dense_supported(int F, int C, int N, int H, int W) {
-    return encode_fn() != nullptr && F >= 1 && C >= 1 && N >= 1 && H >= 1 && W >= 1 && W <= 4096 && H <= 4096;
+    // the layout kernels in front of the GEMM put (image, 64-channel block) on a grid dimension of at most 65535
+    const long long cblocks = (C + kKBlock - 1) / kKBlock;
+    return encode_fn() != nullptr && F >= 1 && C >= 1 && N >= 1 && H >= 1 && W >= 1 && W <= 4096 && H <= 4096 &&
+           N * cblocks <= 65535;
 }
 
 // Pixel box (TW x TH x TN <= 128) that wastes the fewest MMA rows for this image size.

@@ -133,6 +133,18 @@ def test_error_codes(B):
     assert b"permutation" in lib.patdnn_strerror(5)
 
 
+def test_size_limits_are_refused_at_encode_time(B):
+    L = synth.make_layer("lim", F=4, C=4, N=1, H=8, W=8, seed=2, draw_input=False)
+    for kw in (dict(N=1, H=65536, W=8), dict(N=1, H=8, W=65536), dict(N=65536, H=8, W=8),
+               dict(N=1, H=32768, W=32768)):                 # the last: 4 * 2^30 elements in one image
+        with pytest.raises(B.PatdnnError) as e:
+            B.encode(L.weights, L.mask, L.patterns, host_only=True, **kw)
+        assert e.value.status == 2, kw
+    # one image may come close to 2^31 elements, and a batch may hold more than that
+    B.encode(L.weights, L.mask, L.patterns, N=1, H=16384, W=16384, host_only=True).free()
+    B.encode(L.weights, L.mask, L.patterns, N=4096, H=1024, W=1024, host_only=True).free()
+
+
 def test_host_only_handle_refuses_to_run(B):
     L = synth.config1()
     layer = B.encode(L.weights, L.mask, L.patterns, N=1, H=32, W=32, host_only=True)

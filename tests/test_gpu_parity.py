@@ -294,6 +294,36 @@ def test_vgg_full_size_standalone(i, N):
     assert_close(got, oracle_layer(L, x=x), TOL_F32, f"vgg L{i + 1} N={N}")
 
 
+@pytest.mark.parametrize("variant,dtype", [("auto", "f16"), ("tiled", "f16"), ("prun", "f16"), ("auto", "f32")])
+def test_batch_holding_more_than_two_to_the_31_elements(variant, dtype):
+    """64 -> 64 @ 128x128 at batch 2112: input and output hold 2.2e9 elements each, so every offset that includes the
+    image index needs 64 bits.  The first and last images and those on both sides of the 2^32-byte and 2^31-element
+    boundaries (images 1024 and 2048) are compared whole with the oracle."""
+    import oracle
+    import torch
+    from paper_2001_00138_b200 import binding as B
+    N, C, F, H, W = 2112, 64, 64, 128, 128
+    if torch.cuda.mem_get_info()[0] < 40e9:
+        pytest.skip("needs ~30 GB of free device memory")
+    L = synth.make_layer("big", F=F, C=C, N=1, H=H, W=W, seed=4242, prune=0.5, dtype=dtype, bias_std=0.1, draw_input=False)
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    xt = torch.rand((N, C, H, W), device="cuda", dtype=tdt, generator=torch.Generator(device="cuda").manual_seed(11))
+    out = torch.full((N, F, H, W), float("nan"), device="cuda", dtype=tdt)
+    layer = B.encode(L.weights, L.mask, L.patterns, N=N, H=H, W=W, dtype=B.F16 if dtype == "f16" else B.F32, relu=True,
+                     bias=L.bias, variant=VARIANTS[variant])
+    try:
+        layer.conv(xt, out, torch.cuda.current_stream().cuda_stream)
+        layer.check()
+        if variant != "auto":
+            assert layer.plan()["variant"] == VARIANTS[variant]
+    finally:
+        layer.free()
+    sel = [0, 1, 1023, 1024, 2047, 2048, N - 2, N - 1]
+    assert bool(torch.isfinite(out[::97]).all())
+    ref = oracle.conv3x3(xt[sel].float().cpu().numpy(), L.weights, L.mask, L.bias, True)
+    assert_close(out[sel].float().cpu().numpy(), ref, TOL_F16 if dtype == "f16" else TOL_F32, f"big batch {variant}/{dtype}")
+
+
 @pytest.mark.parametrize("ks", [1, 2, 4, 8])
 def test_tensor_core_path_with_cluster_split_of_the_channel_loop(ks, monkeypatch):
     """Small batches split the (channel block, tap) loop over the CTAs of a cluster and sum through distributed shared
