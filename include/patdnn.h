@@ -257,6 +257,9 @@ PATDNN_API int patdnn_plan(patdnn_handle h, patdnn_plan_info *info);
  *                         events between the launches switch off their overlap, so time whole steps with
  *                         patdnn_stack_run
  *   patdnn_stack_out_shape  N, F, H, W of the stack's output
+ *   patdnn_stack_generated  writes to *count how many layers of the stack run code generated for them when the stack
+ *                         was created (few-channel first layers; 0 where the run-time compiler is missing or switched
+ *                         off, in which case the static kernel runs)
  * Errors: E_NULL, E_STACK, E_CUDA, E_NO_DEVICE.
  */
 PATDNN_API int patdnn_stack_create(const patdnn_handle *handles, const int32_t *pool_after, int32_t n, patdnn_stack *out);
@@ -266,6 +269,7 @@ PATDNN_API int patdnn_stack_run_host(patdnn_stack s, const void *in_host, void *
 PATDNN_API int patdnn_stack_submit_host(patdnn_stack s, const void *in_host, void *out_host, void *stream);
 PATDNN_API int patdnn_stack_wait_host(patdnn_stack s);
 PATDNN_API int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, int32_t *W);
+PATDNN_API int patdnn_stack_generated(patdnn_stack s, int32_t *count);
 PATDNN_API int patdnn_stack_free(patdnn_stack s);
 
 /* patdnn_maxpool2x2 -- 2x2 / stride-2 max-pool (floor) on DEVICE NCHW tensors of the given dtype; asynchronous.

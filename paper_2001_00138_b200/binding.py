@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "patdnn_encode", "patdnn_conv", "patdnn_conv_static", "patdnn_conv_host", "patdnn_check", "patdnn_free", "patdnn_export", "patdnn_decode",
     "patdnn_plan", "patdnn_stack_create", "patdnn_stack_run", "patdnn_stack_run_host", "patdnn_stack_out_shape",
     "patdnn_stack_free", "patdnn_stack_submit_host", "patdnn_stack_wait_host", "patdnn_maxpool2x2", "patdnn_launch_count", "patdnn_reset_launch_count", "patdnn_strerror",
-    "patdnn_last_cuda_error", "patdnn_version", "patdnn_debug_wait", "patdnn_stack_run_timed",
+    "patdnn_last_cuda_error", "patdnn_version", "patdnn_debug_wait", "patdnn_stack_run_timed", "patdnn_stack_generated",
 )
 
 
@@ -90,6 +90,7 @@ def load() -> ctypes.CDLL:
     lib.patdnn_stack_submit_host.argtypes = [vp, vp, vp, vp]
     lib.patdnn_stack_wait_host.argtypes = [vp]
     lib.patdnn_stack_out_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 4
+    lib.patdnn_stack_generated.argtypes = [vp, ctypes.POINTER(i32)]
     lib.patdnn_stack_free.argtypes = [vp]
     lib.patdnn_maxpool2x2.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
     lib.patdnn_launch_count.restype = ctypes.c_int64
@@ -247,6 +248,12 @@ class Stack:
         v = [ctypes.c_int32() for _ in range(4)]
         _check(load().patdnn_stack_out_shape(self._h, *[ctypes.byref(x) for x in v]), "patdnn_stack_out_shape")
         return tuple(int(x.value) for x in v)
+
+    def generated(self) -> int:
+        """Number of layers of the stack that run code generated for them at stack creation."""
+        v = ctypes.c_int32()
+        _check(load().patdnn_stack_generated(self._h, ctypes.byref(v)), "patdnn_stack_generated")
+        return int(v.value)
 
     def run(self, x, out, stream: int = 0) -> None:
         _check(load().patdnn_stack_run(self._h, _ptr(x), _ptr(out), stream), "patdnn_stack_run")

@@ -890,6 +890,14 @@ int patdnn_stack_out_shape(patdnn_stack s, int32_t *N, int32_t *F, int32_t *H, i
     return PATDNN_OK;
 }
 
+int patdnn_stack_generated(patdnn_stack s, int32_t *count) {
+    if (!s || !count) return PATDNN_E_NULL;
+    int32_t n = 0;
+    for (const SmallCJit *j : s->smallc_jit) n += j ? 1 : 0;
+    *count = n;
+    return PATDNN_OK;
+}
+
 int patdnn_stack_free(patdnn_stack s) {
     if (!s) return PATDNN_OK;
     for (int b = 0; b < 2; ++b)

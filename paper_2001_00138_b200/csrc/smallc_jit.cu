@@ -98,6 +98,8 @@ std::string hexfloat(float v) {
     return buf;
 }
 
+constexpr int kSplitWarps = 4;                                   // warps per CTA of the split-operand form
+
 // The CUDA C++ source of the layer's kernel.
 // nchw_out: write the caller's NCHW tensor (a layer run on its own) instead of the next layer's split operands.
 std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int C, bool relu, bool half_in, bool nchw_out) {
@@ -117,19 +119,23 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
     }
     std::ostringstream o;
     const int S = half_in ? 1 : 2;
+    // Split-operand form: 4 warps per CTA and the finished 16-byte chunks go to the warp's shared-memory stage group by
+    // group, so that a thread holds only its 3x3xC inputs and eight accumulators (six CTAs per SM); the NCHW form
+    // stores straight from registers.
+    const int warps = nchw_out ? 8 : kSplitWarps;
     o << "typedef unsigned int u32;\n";
-    o << "extern \"C\" __global__ void __launch_bounds__(256, 2) patdnn_first_layer(const "
+    o << "extern \"C\" __global__ void __launch_bounds__(" << warps * 32 << ", " << (nchw_out ? 2 : 6) << ") patdnn_first_layer(const "
       << (half_in ? "unsigned short" : "float") << " *__restrict__ in, "
       << (nchw_out && !half_in ? "float" : "unsigned short") << " *__restrict__ dst, int N, int H, int W) {\n";
-    if (!nchw_out) o << "  __shared__ __align__(16) unsigned char stage[8][32 * 128];\n";
+    if (!nchw_out) o << "  __shared__ __align__(16) unsigned char stage[" << warps << "][" << S << "][32 * 128];\n";
     o << "  asm volatile(\"griddepcontrol.launch_dependents;\" ::: \"memory\");\n";
     o << "  asm volatile(\"griddepcontrol.wait;\" ::: \"memory\");\n";
     o << "  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;\n";
     o << "  const unsigned P = (unsigned)N * H * W;\n";
     o << "  const size_t plane_out = (size_t)P * 64;\n";
-    if (!nchw_out) o << "  unsigned char *st = stage[warp];\n";
+    if (!nchw_out) o << "  unsigned char *st = stage[warp][0];\n";
     else o << "  (void)warp;\n";
-    o << "  for (unsigned p0 = (blockIdx.x * 8 + warp) * 32; p0 < P; p0 += gridDim.x * 8 * 32) {\n";
+    o << "  for (unsigned p0 = (blockIdx.x * " << warps << " + warp) * 32; p0 < P; p0 += gridDim.x * " << warps << " * 32) {\n";
     o << "    const unsigned pix = p0 + lane; const bool ok = pix < P;\n";
     o << "    const unsigned q = ok ? pix : 0u, r_ = q / (unsigned)W; const int x = (int)(q - r_ * W);\n";
     o << "    const unsigned n = r_ / (unsigned)H; const int y = (int)(r_ - n * H);\n";
@@ -145,8 +151,7 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
     else
         o << "            t = base[c * plane + (dy - 1) * W + (dx - 1)];\n";
     o << "          }\n          v[9 * c + 3 * dy + dx] = t;\n        }\n";
-    if (!nchw_out) o << "    u32 hi[32]" << (S == 2 ? ", lo[32]" : "") << ";\n";
-    else o << "    const size_t obase = (size_t)n * " << fkw.F << " * plane + (size_t)y * W + x;\n";
+    if (nchw_out) o << "    const size_t obase = (size_t)n * " << fkw.F << " * plane + (size_t)y * W + x;\n";
     for (int g = 0; g < 8; ++g) {
         o << "    {\n";
         for (int j = 0; j < 8; ++j) o << "      float a" << j << " = " << hexfloat(b[8 * g + j]) << ";\n";
@@ -172,32 +177,36 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
             o << "    }\n";
             continue;
         }
+        o << "      u32 h0, h1, h2, h3" << (S == 2 ? ", l0, l1, l2, l3" : "") << ";\n";
         for (int j = 0; j < 8; j += 2) {
-            const int w = (8 * g + j) / 2;
+            const int w = j / 2;
             if (S == 2) {
-                o << "      { u32 h; asm(\"cvt.rn.bf16x2.f32 %0, %1, %2;\" : \"=r\"(h) : \"f\"(a" << j + 1 << "), \"f\"(a" << j << "));\n"
-                  << "        const float e0 = a" << j << " - __uint_as_float(h << 16), e1 = a" << j + 1 << " - __uint_as_float(h & 0xffff0000u);\n"
-                  << "        u32 l; asm(\"cvt.rn.bf16x2.f32 %0, %1, %2;\" : \"=r\"(l) : \"f\"(e1), \"f\"(e0));\n"
-                  << "        hi[" << w << "] = h; lo[" << w << "] = l; }\n";
+                o << "      asm(\"cvt.rn.bf16x2.f32 %0, %1, %2;\" : \"=r\"(h" << w << ") : \"f\"(a" << j + 1 << "), \"f\"(a" << j << "));\n"
+                  << "      { const float e0 = a" << j << " - __uint_as_float(h" << w << " << 16), e1 = a" << j + 1 << " - __uint_as_float(h" << w
+                  << " & 0xffff0000u);\n"
+                  << "        asm(\"cvt.rn.bf16x2.f32 %0, %1, %2;\" : \"=r\"(l" << w << ") : \"f\"(e1), \"f\"(e0)); }\n";
             } else {
-                o << "      { u32 h; asm(\"cvt.rn.f16x2.f32 %0, %1, %2;\" : \"=r\"(h) : \"f\"(a" << j + 1 << "), \"f\"(a" << j << "));\n"
-                  << "        hi[" << w << "] = h; }\n";
+                o << "      asm(\"cvt.rn.f16x2.f32 %0, %1, %2;\" : \"=r\"(h" << w << ") : \"f\"(a" << j + 1 << "), \"f\"(a" << j << "));\n";
             }
         }
+        // this group's eight filters are 16-byte chunk g of the pixel's 128-byte row (chunk index swizzled by the row)
+        o << "      *reinterpret_cast<uint4 *>(st + lane * 128 + ((" << g << " ^ (lane & 7)) << 4)) = make_uint4(h0, h1, h2, h3);\n";
+        if (S == 2)
+            o << "      *reinterpret_cast<uint4 *>(st + 4096 + lane * 128 + ((" << g << " ^ (lane & 7)) << 4)) = make_uint4(l0, l1, l2, l3);\n";
         o << "    }\n";
     }
     if (!nchw_out) o << "    const int rows = (int)(P - p0 < 32u ? P - p0 : 32u);\n";
+    if (!nchw_out) o << "    __syncwarp();\n";
     for (int sp = 0; sp < (nchw_out ? 0 : S); ++sp) {
-        const char *arr = sp == 0 ? "hi" : "lo";
-        o << "    __syncwarp();\n#pragma unroll\n    for (int ch = 0; ch < 8; ++ch)\n"
-          << "      *reinterpret_cast<uint4 *>(st + lane * 128 + ((ch ^ (lane & 7)) << 4)) = make_uint4(" << arr << "[4 * ch], " << arr
-          << "[4 * ch + 1], " << arr << "[4 * ch + 2], " << arr << "[4 * ch + 3]);\n"
-          << "    __syncwarp();\n    {\n      unsigned char *g = reinterpret_cast<unsigned char *>(dst + " << sp
+        o << "    {\n      unsigned char *g = reinterpret_cast<unsigned char *>(dst + " << sp
           << " * plane_out + (size_t)p0 * 64);\n#pragma unroll\n      for (int k = 0; k < 8; ++k) {\n"
           << "        const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;\n"
-          << "        if (row < rows) *reinterpret_cast<uint4 *>(g + idx * 16) = *reinterpret_cast<const uint4 *>(st + row * 128 + ((ch ^ (row & 7)) << 4));\n"
+          << "        if (row < rows) *reinterpret_cast<uint4 *>(g + idx * 16) = *reinterpret_cast<const uint4 *>(st + " << sp * 4096
+          << " + row * 128 + ((ch ^ (row & 7)) << 4));\n"
           << "      }\n    }\n";
     }
+    if (!nchw_out) o << "    __syncwarp();\n";                  // the stage is free again before the next pixels' chunks
+
     o << "  }\n}\n";
     return o.str();
 }
@@ -207,6 +216,7 @@ std::string generate_source(const Fkw &fkw, const std::vector<float> &bias, int 
 struct SmallCJit {
     CUmodule mod = nullptr;
     CUfunction fn = nullptr;
+    int warps = 8;                                               // warps per CTA the source was generated for
 };
 
 SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int C, int relu, int is_half, std::string *log,
@@ -246,18 +256,21 @@ SmallCJit *smallc_jit_build(const Fkw &fkw, const std::vector<float> &bias, int 
         if (log) *log = "cuModuleLoadData failed";
         return nullptr;
     }
+    j->warps = nchw_out ? 8 : kSplitWarps;
     return j;
 }
 
 cudaError_t smallc_jit_launch(SmallCJit *j, const void *in, void *dst, int N, int H, int W, cudaStream_t st) {
     const long long P = static_cast<long long>(N) * H * W;
     if (P == 0) return cudaSuccess;
-    const long long blocks_needed = (P + 255) / 256;
-    const unsigned grid = static_cast<unsigned>(blocks_needed < sm_count() * 8 ? blocks_needed : sm_count() * 8);
+    const int per_cta = j->warps * 32;
+    const long long blocks_needed = (P + per_cta - 1) / per_cta;
+    const long long cap = static_cast<long long>(sm_count()) * (2048 / per_cta);   // a few rounds of resident CTAs
+    const unsigned grid = static_cast<unsigned>(blocks_needed < cap ? blocks_needed : cap);
     CUlaunchConfig cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDimX = grid; cfg.gridDimY = 1; cfg.gridDimZ = 1;
-    cfg.blockDimX = 256; cfg.blockDimY = 1; cfg.blockDimZ = 1;
+    cfg.blockDimX = static_cast<unsigned>(per_cta); cfg.blockDimY = 1; cfg.blockDimZ = 1;
     cfg.sharedMemBytes = 0;
     cfg.hStream = st;
     CUlaunchAttribute attr[1];

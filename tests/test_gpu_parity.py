@@ -158,6 +158,7 @@ def test_few_channel_first_layer_writes_the_next_layers_operands(shape, dtype, g
         mid = mid.astype(np.float16).astype(np.float32)          # the layer boundary stores fp16
     ref = oracle.conv3x3(mid, L1.weights, L1.mask, L1.bias, False)
     stack = B.Stack([h0, h1], [0, 0])
+    assert stack.generated() == (1 if generated else 0), "the generated kernel must be the one that runs (no silent fallback)"
     out = torch.empty((N, 48, H, W), device="cuda", dtype=tdt)
     B.reset_launch_count()
     stack.run(torch.from_numpy(L0.x).to("cuda", dtype=tdt), out, torch.cuda.current_stream().cuda_stream)

@@ -138,6 +138,7 @@ def test_benchmark_stack_whole_images_against_the_chained_oracle(N):
     handles = [B.encode(L.weights, L.mask, L.patterns, N=N, H=L.H, W=L.W, relu=True, bias=L.bias) for L in layers]
     pools = [1 if i in synth.VGG16_POOL_AFTER else 0 for i in range(13)]
     stack = B.Stack(handles, pools)
+    assert stack.generated() == 1, "the RGB layer runs the code generated for it, as in the benchmark"
     x = synth.vgg16_input(N)
     out = torch.full(stack.out_shape(), float("nan"), device="cuda")
     stack.run(torch.from_numpy(x).cuda(), out, torch.cuda.current_stream().cuda_stream)
