@@ -435,6 +435,17 @@ def suite_dense_context(synth, torch):
                               "library": "torch.nn.functional.conv2d (cuDNN), fp32, TF32 off"}), flush=True)
 
 
+def workload_config(batch: int) -> dict:
+    """The `config` object of the JSON line: the workload both arms are quoted on."""
+    return {"workload": f"vgg16_3x3_stack_n{batch}", "batch_per_gpu": batch, "layers": 13,
+            "patterns": 8, "connectivity_pruning": "0% layer 1, 60% layers 2-13",
+            "l2": ("working set larger than L2 (first activation alone is %d MB); input buffers rotated"
+                   % (batch * 64 * 224 * 224 * 4 // 2**20)) if batch >= 8 else "see batch1 leg",
+            "step": "13 conv layers chained by the library: RGB layer as FP32 code generated for it, 12 tensor-core GEMM "
+                    "layers (some with a K-split tail launch), every kernel writing the next layer's operands directly; "
+                    "the 4 max-pools are taken in epilogues"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -453,7 +464,7 @@ def run_reference(args):
         "impl": "reference", "metric": "effective GFLOP/s on nonzero MACs, pattern-sparse 3x3 conv", "value": val,
         "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"vgg16_3x3_stack_n{args.batch}", "sample": sample},
+        "config": workload_config(args.batch),            # the GPU arm's configuration; what one step samples of it: `sample`
         "cpu_baseline": {"value": val, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -464,7 +475,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=32)
@@ -690,13 +701,7 @@ def main():
         "value": replicas.whole_job_value(r["flops"], ms * 1e-3, world) / 1e9,
         "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"vgg16_3x3_stack_n{args.batch}", "batch_per_gpu": args.batch, "layers": 13,
-                   "patterns": 8, "connectivity_pruning": "0% layer 1, 60% layers 2-13",
-                   "l2": "working set larger than L2 (first activation alone is %d MB); input buffers rotated"
-                         % (args.batch * 64 * 224 * 224 * 4 // 2**20) if args.batch >= 8 else "see batch1 leg",
-                   "step": "13 conv layers chained by the library: RGB layer as FP32 code generated for it, 12 tensor-core GEMM "
-                           "layers (some with a K-split tail launch), every kernel writing the next layer's operands directly; "
-                           "the 4 max-pools are taken in epilogues"},
+        "config": workload_config(args.batch),
         "clocks": r["clocks"],
         "e2e": {"value": world * r["flops"] / (e2e_ms * 1e-3) / 1e9, "unit": "GFLOP/s",
                 "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "ms_per_step": e2e_ms,
