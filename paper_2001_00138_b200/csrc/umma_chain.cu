@@ -20,7 +20,7 @@
 //
 // Every wait is bounded -- mbarrier waits as in the other kernels, the grid barrier by the same polling budget -- and a
 // wait that runs out records a status word, after which every role of every CTA falls through to the common exit.
-// The launch is cooperative, so all CTAs are resident together; no cluster, no multicast.
+// The launch is cooperative, so all CTAs are resident together; no clusters, every CTA loads its own operands.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
