@@ -31,9 +31,11 @@ FP32_LANES = 128                      # FP32 FMA lanes per SM on this architectu
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (conv_umma_halo_kernel on the
 # 256 -> 256 @ 56x56 layer): 28.5 MB in the ncu capture at batch 8 (profiles/conv_umma_halo_kernel_vgg16_L06_n8.txt),
 # scaled by the units of a batch-32 launch (x4; reads grow in proportion, the output additionally leaves L2 at that size)
-TRAFFIC_BYTES_PER_LAUNCH = 4 * (28093696 + 267776)
-TRAFFIC_NOTE = ("dominant kernel (conv_umma_halo_kernel, 256 -> 256 @ 56x56): ncu capture at batch 8 scaled x4 to the "
-                "batch-32 launch (extrapolated; algorithmic bytes of that launch: 112.5 MB in + 2.4 MB weights)")
+TRAFFIC_BYTES_PER_LAUNCH = 104771072 + 52571392
+TRAFFIC_NOTE = ("dominant kernel (conv_umma_halo_kernel, 256 -> 256 @ 56x56, the form it has inside the stack): "
+                "dram__bytes_read + dram__bytes_write of one launch at the benchmark's batch 32, one ncu capture "
+                "(profiles/conv_umma_halo_kernel_vgg16_L06_n32.txt); algorithmic bytes of that launch: 102.8 MB split input + "
+                "2.4 MB weights + 102.8 MB output, of which ~50 MB were still in L2 when the kernel ended")
 
 
 def alu_peak_tflops(torch=None):
